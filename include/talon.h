@@ -1,0 +1,199 @@
+/*
+ * talon.h -- C ABI of the B200 (sm_100a) hot path of Talon, the confidence-aware,
+ * budget-driven speculative-decoding method.
+ *
+ * The library builds a draft token tree layer by layer under a fixed node budget
+ * (Algorithm 2 of the paper: Top-K at the root, Eq. 5; confidence gate p(u) >= mu * m_d
+ * below it, Eq. 3-4; truncation to the remaining budget) and verifies it: tree attention
+ * under the ancestor mask followed by the greedy longest-accepted-path walk (Appendix B).
+ * The draft and target model forwards are the caller's: the caller hands in their logits
+ * and the projected Q/K/V.
+ *
+ * Conventions that hold for every call unless a comment says otherwise:
+ *  - Pointers named in a "device" comment are CUDA device pointers owned by the caller.
+ *    The library never frees or reallocates them.  "host" pointers are ordinary memory.
+ *  - A call only enqueues work on `stream` (a cudaStream_t passed as void*) and returns;
+ *    it performs no synchronisation and no allocation after talon_create
+ *    (talon_step_host and talon_poll_status are the two documented exceptions).
+ *  - Errors that the host can see (null pointer, size out of range, misalignment) return
+ *    a status at once with nothing enqueued.  Errors only the device can see (NaN or +inf
+ *    logit, a row of only -inf) set a device status word that talon_poll_status reads;
+ *    outputs stay defined (the layer adds no node for the affected sequence).
+ *  - One context serves one stream at a time; calls on one context must not overlap.
+ *  - Sequences of a batch are independent.  B is fixed by talon_reset until the next reset.
+ *
+ * Notation: B batch, V vocabulary, N node budget (root included, <= 128), K root top-k,
+ * k per-parent candidate cap, D_max depth cap, W = ceil(N/64) mask words, Hq/Hkv query
+ * and key/value heads, g = Hq/Hkv, Dh = 128 head dimension, L_b prefix length.
+ */
+#ifndef TALON_H_
+#define TALON_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct talon_ctx talon_ctx;
+
+typedef enum {
+  TALON_OK = 0,
+  TALON_ERR_INVALID_ARG = 1, /* null pointer, size out of range, misaligned row          */
+  TALON_ERR_CAPACITY = 2,    /* request exceeds what the context was created for          */
+  TALON_ERR_CUDA = 3,        /* a CUDA runtime call failed (see stderr for the message)   */
+  TALON_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up                        */
+  TALON_ERR_NONFINITE = 5,   /* NaN / +inf logit, or a row holding only -inf              */
+  TALON_ERR_UNSUPPORTED = 6  /* valid in the paper, not built (e.g. head_dim != 128)      */
+} talon_status;
+
+/* Hyper-parameters of Algorithm 2 ("Require" line: budget N, width K, threshold mu) plus the
+ * shapes the verification step needs.  Defaults of the paper: N = 60, K = 10, mu = 0.03. */
+typedef struct {
+  int32_t batch_max;   /* largest B any later call may use (1..1024)                         */
+  int32_t vocab;       /* V (2 .. 2^24-1)                                                    */
+  int32_t budget;      /* N, root included (2..128)                                          */
+  int32_t root_topk;   /* K of Eq. 5 (1..128)                                                */
+  int32_t cand_topk;   /* k: candidates kept per parent before pooling (1..128); 0 = N-1,    *
+                        * which reproduces Eq. 3's whole-vocabulary pool exactly, because a  *
+                        * parent can never place more than N-|T| children                   */
+  int32_t max_depth;   /* D_max: no node deeper than this (1..126)                           */
+  int32_t init_layers; /* leading layers that use Top-K instead of the gate; paper: 1        */
+  int32_t n_q_heads;   /* Hq                                                                 */
+  int32_t n_kv_heads;  /* Hkv, divides Hq                                                    */
+  int32_t head_dim;    /* Dh, must be 128                                                    */
+  double  mu;          /* gate threshold of Eq. 4, in (0, 1]                                 */
+} talon_params;
+
+/* The draft tree T of Algorithm 2 as flat per-sequence arrays in caller-owned DEVICE memory.
+ * Node 0 is the root x_t; nodes are stored layer by layer, each layer sorted by
+ * (parent index, token id), so parent[i] < i.  Slots n_nodes[b]..N-1 hold sentinels after
+ * talon_build_tree (token = parent = depth = position = -1, score = -inf, mask = own bit). */
+typedef struct {
+  int32_t  *n_nodes;   /* [B]              |T| per sequence                                  */
+  int32_t  *token;     /* [B, N]           token id of each node                             */
+  int32_t  *parent;    /* [B, N]           parent node index, -1 for the root                */
+  int32_t  *depth;     /* [B, N]           root = 0                                          */
+  int32_t  *position;  /* [B, N]           prefix_len + depth (written by talon_build_tree)  */
+  int32_t  *layer_off; /* [B, D_max + 2]   nodes of depth d are layer_off[d]..layer_off[d+1]-1 */
+  double   *score;     /* [B, N]           log of Eq. 2's path probability p(v)              */
+  uint64_t *mask;      /* [B, N, W]        bit j of row i set iff node i attends to node j
+                        *                  (itself and its ancestors; Fig. 2(b), Appendix B)  */
+} talon_tree;
+
+/* How talon_expand_layer finds the logit row of a frontier node. */
+enum {
+  TALON_ROWS_BY_NODE = 0,  /* row index = b * rows_per_seq + node index                       */
+  TALON_ROWS_PACKED  = 1   /* row index = b * rows_per_seq + (node index - first frontier node) */
+};
+
+/* Creates a context on CUDA device `device` and allocates its workspace there (the only
+ * allocation the library makes, apart from talon_step_host's staging buffers).
+ * Returns INVALID_ARG / UNSUPPORTED for out-of-range parameters, CUDA on allocation failure. */
+talon_status talon_create(talon_ctx **out_ctx, const talon_params *params, int device);
+
+/* Frees the context's workspace.  Caller memory is untouched.  Null is accepted. */
+talon_status talon_destroy(talon_ctx *ctx);
+
+/* Algorithm 2, lines 1-2: T <- {x_t}, P_0 <- {x_t}, p(x_t) <- 1, d <- 0, for B sequences.
+ * root_tok   device [B]  last committed token x_t of each sequence
+ * prefix_len device [B]  number of tokens before x_t, i.e. the KV-cache length L_b (>= 0)
+ * Clears the device status word. */
+talon_status talon_reset(talon_ctx *ctx, const talon_tree *tree, const int32_t *root_tok,
+                         const int32_t *prefix_len, int32_t B, void *stream);
+
+/* One pass of Algorithm 2's while-body for every sequence that still has budget: reads the
+ * draft logits of the current frontier P_d (all nodes of depth d), forms the candidate pool
+ * S_d with path scores p(u) = p(v) * softmax(logits_v)[w] (Eq. 3; per-parent top-k first),
+ * applies Top-K (d < init_layers, Eq. 5) or the gate p(u) >= mu * max p (Eq. 4), truncates
+ * to the remaining budget by score, and appends the survivors as depth d+1.
+ * Ties: higher score first, then lower parent index, then lower token id.
+ * logits       device fp32; row r starts at logits + r * row_stride; 16-byte aligned
+ * row_stride   elements between rows, a multiple of 4 and >= V
+ * rows_per_seq rows reserved per sequence in `logits` (N for BY_NODE)
+ * layout       TALON_ROWS_BY_NODE or TALON_ROWS_PACKED
+ * A sequence whose tree is full, whose frontier is empty, or whose depth reached D_max is
+ * left unchanged; once d == D_max the call is a no-op.  -inf logits are legal (p = 0,
+ * never selected).  The number of calls since talon_reset is the layer index d. */
+talon_status talon_expand_layer(talon_ctx *ctx, const talon_tree *tree, const float *logits,
+                                int64_t row_stride, int32_t rows_per_seq, int32_t layout,
+                                void *stream);
+
+/* Number of talon_expand_layer calls since the last talon_reset (host counter). */
+int32_t talon_layers_run(const talon_ctx *ctx);
+
+/* Closes the tree for verification (Fig. 2(b), Appendix B): position = prefix_len + depth,
+ * sentinels in unused slots, remaining layer_off entries = n_nodes.
+ * dense_mask  device [B, N, N] uint8 or null: if given, receives the mask as bytes
+ *             (1 = row node attends to column node). */
+talon_status talon_build_tree(talon_ctx *ctx, const talon_tree *tree, uint8_t *dense_mask,
+                              void *stream);
+
+/* Tree attention of the verification forward (Appendix B): query node i of sequence b and
+ * query head h attends to all L_b prefix keys and to the tree keys j with mask bit (i, j)
+ * set, softmax(sm_scale * q.k) in fp32, times V, accumulated in fp32, written as bf16.
+ * All tensors bf16, device memory:
+ *  q        [B, N, Hq, Dh] contiguous
+ *  k_prefix, v_prefix  token t, head h of sequence b at
+ *           base + (kv_start[b] + t) * kv_stride_t + h * kv_stride_h   (elements; Dh contiguous;
+ *           strides multiples of 8)
+ *  k_tree, v_tree      [B, N, Hkv, Dh] contiguous: keys/values of the tree tokens themselves
+ *  kv_start device [B] int64 token offsets of each sequence's block (ragged or padded)
+ *  max_prefix_len      host upper bound of the prefix lengths given to talon_reset
+ *  out      [B, N, Hq, Dh] contiguous; rows of unused node slots are written as zeros
+ * Rotary embedding is the caller's business: Q/K arrive already rotated. */
+talon_status talon_tree_attention(talon_ctx *ctx, const talon_tree *tree, const void *q,
+                                  const void *k_prefix, const void *v_prefix,
+                                  const void *k_tree, const void *v_tree,
+                                  const int64_t *kv_start, int64_t kv_stride_t,
+                                  int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale,
+                                  void *out, void *stream);
+
+/* Greedy verification (Appendix B steps 1-2 at temperature 0): t_i = argmax of the target
+ * logits after node i (lowest id among equal maxima), then from the root follow the child
+ * whose token equals t_cur until none does.
+ * target_logits device fp32, row of node i of sequence b at (b*N + i) * row_stride; 16-byte aligned rows
+ * target_tok    device [B, N] or null: receives t_i (-1 for unused slots)
+ * accept_len    device [B]: number of accepted draft tokens (root not counted)
+ * accept_nodes  device [B, D_max + 1]: accepted node indices, root first, -1 padded
+ * bonus_tok     device [B]: target token after the last accepted node */
+talon_status talon_accept(talon_ctx *ctx, const talon_tree *tree, const float *target_logits,
+                          int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
+                          int32_t *accept_nodes, int32_t *bonus_tok, void *stream);
+
+/* Synchronises `stream`, reads and returns the device status word (OK, NONFINITE, TIMEOUT,
+ * CAPACITY).  The word stays set until the next talon_reset. */
+talon_status talon_poll_status(talon_ctx *ctx, void *stream);
+
+/* Host buffers in, host results out: one whole draft-and-verify step (reset, up to D_max
+ * expansion layers, build, tree attention, accept) with the host-to-device and
+ * device-to-host copies included.  All pointers are HOST memory (pinned memory makes the
+ * copies asynchronous).  Layouts as in the device calls with rows BY_NODE and dense tensors:
+ *  draft_logits  [B, N, V] fp32: row i holds the draft logits of node i (rows of nodes that
+ *                are never expanded are not read)
+ *  target_logits [B, N, V] fp32
+ *  q [B,N,Hq,Dh], k_prefix/v_prefix [sum_b L_b, Hkv, Dh] (sequences back to back),
+ *  k_tree/v_tree [B,N,Hkv,Dh], all bf16
+ *  outputs: out_attn [B,N,Hq,Dh] bf16 (may be null), n_nodes [B], token/parent/depth/position
+ *  [B,N] (each may be null), accept_len [B], accept_nodes [B, D_max+1], bonus_tok [B].
+ * The first call allocates device staging buffers sized for batch_max inside the context
+ * (a later call with a longer total prefix reallocates).  Synchronises `stream` before
+ * returning and returns the device status. */
+talon_status talon_step_host(talon_ctx *ctx, int32_t B, const int32_t *root_tok,
+                             const int32_t *prefix_len, const float *draft_logits,
+                             const float *target_logits, const void *q, const void *k_prefix,
+                             const void *v_prefix, const void *k_tree, const void *v_tree,
+                             float sm_scale, void *out_attn, int32_t *n_nodes, int32_t *token,
+                             int32_t *parent, int32_t *depth, int32_t *position,
+                             int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                             void *stream);
+
+/* Number of kernels the library has launched through this context since creation. */
+int64_t talon_launch_count(const talon_ctx *ctx);
+
+const char *talon_status_string(talon_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TALON_H_ */

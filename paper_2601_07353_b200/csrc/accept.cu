@@ -1,0 +1,162 @@
+// Greedy verification (Appendix B of the paper, steps 1-2 at temperature 0) for sm_100a.
+//
+//   target_argmax_kernel : t_i = argmax_w target_logits[b, i, w] for every tree node, one
+//                          streaming pass with 128-bit loads.  Rows are cut into chunks so
+//                          that a single sequence still fills the GPU; chunks meet in a
+//                          64-bit atomicMax on a packed (logit, lowest-token-first) key.
+//   accept_walk_kernel   : decodes the keys, then walks from the root along the child whose
+//                          token equals the target's choice until none does.
+#include <math_constants.h>
+
+#include "talon_internal.cuh"
+
+namespace talon {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+
+struct ArgmaxArgs {
+  const float *logits;
+  int64_t row_stride;
+  const int32_t *n_nodes;
+  int B, N, V;
+  int splits, chunk_len;
+  unsigned long long *best;   // [B*N], zero on entry
+  int *status;
+};
+
+__global__ void __launch_bounds__(EXP_THREADS)
+target_argmax_kernel(ArgmaxArgs a) {
+  __shared__ unsigned long long s_key[EXP_WARPS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_items = a.B * a.N * a.splits;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int row = item / a.splits, chunk = item - row * a.splits;
+    const int b = row / a.N, i = row - b * a.N;
+    if (i >= a.n_nodes[b]) continue;                       // unused node slot (CTA-uniform)
+    const float *rowp = a.logits + (int64_t)row * a.row_stride;
+    const int start = chunk * a.chunk_len;
+    const int end = min(a.V, start + a.chunk_len);
+    float bestv = -CUDART_INF_F;
+    uint32_t besti = 0xFFFFFFFFu;
+    bool bad = false;
+    for (int base = start; base < end; base += EXP_TILE) {
+      float v[EXP_UNROLL][EXP_VEC];
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u) {
+        const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+        if (idx + EXP_VEC <= end) {
+          const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
+          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+        } else {
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u) {
+        const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+#pragma unroll
+        for (int e = 0; e < EXP_VEC; ++e) {
+          const float x = v[u][e];
+          bad |= (x != x);
+          // strict > keeps the lowest index among equal values; the first in-range element
+          // claims the slot even if it is -inf
+          if (idx + e < end && (x > bestv || besti == 0xFFFFFFFFu)) { bestv = x; besti = (uint32_t)(idx + e); }
+        }
+      }
+    }
+    unsigned long long key = (besti == 0xFFFFFFFFu) ? 0ull : cand_key(bestv, besti);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(FULL, key, o);
+      key = other > key ? other : key;
+    }
+    if (__any_sync(FULL, bad) && lane == 0) atomicOr(a.status, STATUS_NONFINITE);
+    __syncthreads();
+    if (lane == 0) s_key[warp] = key;
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long k = s_key[0];
+      for (int w = 1; w < EXP_WARPS; ++w) k = s_key[w] > k ? s_key[w] : k;
+      if (a.splits == 1) a.best[row] = k;
+      else atomicMax(&a.best[row], k);
+    }
+  }
+}
+
+struct WalkArgs {
+  talon_tree t;
+  int lo_stride;
+  int B, N, max_depth;
+  unsigned long long *best;
+  int32_t *target_tok;      // [B*N] workspace or caller buffer
+  int32_t *accept_len, *accept_nodes, *bonus_tok;
+};
+
+// one warp per sequence
+__global__ void accept_walk_kernel(WalkArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (b >= a.B) return;
+  const size_t nb = (size_t)b * a.N;
+  const int n = a.t.n_nodes[b];
+  for (int i = lane; i < a.N; i += 32) {
+    const unsigned long long k = a.best[nb + i];
+    a.best[nb + i] = 0ull;                                  // leave the workspace clean
+    a.target_tok[nb + i] = (i < n && k != 0ull) ? (int32_t)key_tok(k) : -1;
+  }
+  __syncwarp();
+  int cur = 0, len = 0;
+  if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1)] = 0;
+  for (int d = 0; d < a.max_depth; ++d) {
+    const int want = a.target_tok[nb + cur];
+    const int lo = a.t.layer_off[b * a.lo_stride + d + 1];
+    const int hi = a.t.layer_off[b * a.lo_stride + d + 2];
+    int found = -1;
+    for (int c0 = lo; c0 < hi; c0 += 32) {
+      const int c = c0 + lane;
+      const bool hit = c < hi && a.t.parent[nb + c] == cur && a.t.token[nb + c] == want;
+      const unsigned m = __ballot_sync(FULL, hit);
+      if (m) { found = c0 + __ffs(m) - 1; break; }
+    }
+    if (found < 0) break;
+    cur = found;
+    ++len;
+    if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1) + len] = cur;
+  }
+  for (int i = len + 1 + lane; i <= a.max_depth; i += 32) a.accept_nodes[(size_t)b * (a.max_depth + 1) + i] = -1;
+  if (lane == 0) {
+    a.accept_len[b] = len;
+    a.bonus_tok[b] = a.target_tok[nb + cur];
+  }
+}
+
+talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                           int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
+                           int32_t *bonus_tok, cudaStream_t st) {
+  const int rows = c->B * c->p.budget;
+  const LayerGeom g = make_geom(rows, c->p.vocab, c->exp_grid);
+  ArgmaxArgs aa;
+  aa.logits = target_logits; aa.row_stride = row_stride; aa.n_nodes = t->n_nodes;
+  aa.B = c->B; aa.N = c->p.budget; aa.V = c->p.vocab;
+  aa.splits = g.splits; aa.chunk_len = g.chunk_len;
+  aa.best = c->d_argmax; aa.status = c->d_status;
+  long long items = (long long)rows * g.splits;
+  int grid = c->exp_grid;
+  if (items < grid) grid = (int)items;
+  target_argmax_kernel<<<grid, EXP_THREADS, 0, st>>>(aa);
+  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+
+  WalkArgs wa;
+  wa.t = *t; wa.lo_stride = c->p.max_depth + 2;
+  wa.B = c->B; wa.N = c->p.budget; wa.max_depth = c->p.max_depth;
+  wa.best = c->d_argmax; wa.target_tok = target_tok ? target_tok : c->d_target_tok;
+  wa.accept_len = accept_len; wa.accept_nodes = accept_nodes; wa.bonus_tok = bonus_tok;
+  const int warps_per_block = 4;
+  accept_walk_kernel<<<(c->B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(wa);
+  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+  c->launches += 2;
+  return TALON_OK;
+}
+
+}  // namespace talon

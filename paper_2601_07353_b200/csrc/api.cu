@@ -1,0 +1,339 @@
+// C ABI of libtalon: argument checks, context life cycle, and the host-buffer step.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "talon_internal.cuh"
+
+namespace talon {
+talon_status expand_setup(talon_ctx *c);
+talon_status attention_mma_setup();
+}  // namespace talon
+
+// Device staging for talon_step_host.
+struct HostStage {
+  int batch = 0;
+  int64_t prefix_tokens = 0;
+  float *draft = nullptr, *target = nullptr;
+  void *q = nullptr, *kp = nullptr, *vp = nullptr, *kt = nullptr, *vt = nullptr, *out = nullptr;
+  int32_t *root = nullptr, *plen = nullptr;
+  int64_t *kv_start = nullptr;
+  talon_tree tree{};
+  int32_t *accept_len = nullptr, *accept_nodes = nullptr, *bonus = nullptr;
+  int64_t *h_kv_start = nullptr;   // pinned host scratch
+};
+
+#define TALON_CUDA_OK(expr)                                                              \
+  do {                                                                                   \
+    cudaError_t e_ = (expr);                                                             \
+    if (e_ != cudaSuccess) {                                                             \
+      std::fprintf(stderr, "talon: %s failed: %s\n", #expr, cudaGetErrorString(e_));     \
+      return TALON_ERR_CUDA;                                                             \
+    }                                                                                    \
+  } while (0)
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static bool tree_complete(const talon_tree *t) {
+  return t && t->n_nodes && t->token && t->parent && t->depth && t->position && t->layer_off && t->score &&
+         t->mask;
+}
+
+static void free_stage(HostStage *s) {
+  if (!s) return;
+  cudaFree(s->draft); cudaFree(s->target); cudaFree(s->q); cudaFree(s->kp); cudaFree(s->vp);
+  cudaFree(s->kt); cudaFree(s->vt); cudaFree(s->out); cudaFree(s->root); cudaFree(s->plen);
+  cudaFree(s->kv_start);
+  cudaFree(s->tree.n_nodes); cudaFree(s->tree.token); cudaFree(s->tree.parent); cudaFree(s->tree.depth);
+  cudaFree(s->tree.position); cudaFree(s->tree.layer_off); cudaFree(s->tree.score); cudaFree(s->tree.mask);
+  cudaFree(s->accept_len); cudaFree(s->accept_nodes); cudaFree(s->bonus);
+  if (s->h_kv_start) cudaFreeHost(s->h_kv_start);
+  delete s;
+}
+
+extern "C" {
+
+const char *talon_status_string(talon_status s) {
+  switch (s) {
+    case TALON_OK: return "ok";
+    case TALON_ERR_INVALID_ARG: return "invalid argument";
+    case TALON_ERR_CAPACITY: return "capacity exceeded";
+    case TALON_ERR_CUDA: return "CUDA runtime error";
+    case TALON_ERR_TIMEOUT: return "device-side wait timed out";
+    case TALON_ERR_NONFINITE: return "non-finite logits";
+    case TALON_ERR_UNSUPPORTED: return "unsupported configuration";
+  }
+  return "unknown status";
+}
+
+talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device) {
+  if (!out_ctx || !p) return TALON_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  if (p->batch_max < 1 || p->batch_max > talon::MAX_BATCH) return TALON_ERR_INVALID_ARG;
+  if (p->vocab < 2 || p->vocab >= (1 << 24)) return TALON_ERR_INVALID_ARG;
+  if (p->budget < 2 || p->budget > talon::MAX_BUDGET) return TALON_ERR_INVALID_ARG;
+  if (p->root_topk < 1 || p->root_topk > 128) return TALON_ERR_INVALID_ARG;
+  if (p->cand_topk < 0 || p->cand_topk > 128) return TALON_ERR_INVALID_ARG;
+  if (p->max_depth < 1 || p->max_depth > 126) return TALON_ERR_INVALID_ARG;
+  if (p->init_layers < 0) return TALON_ERR_INVALID_ARG;
+  if (!(p->mu > 0.0) || !(p->mu <= 1.0)) return TALON_ERR_INVALID_ARG;
+  if (p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads) return TALON_ERR_INVALID_ARG;
+  if (p->head_dim != 128) return TALON_ERR_UNSUPPORTED;
+
+  int n_dev = 0;
+  TALON_CUDA_OK(cudaGetDeviceCount(&n_dev));
+  if (device < 0 || device >= n_dev) return TALON_ERR_INVALID_ARG;
+  TALON_CUDA_OK(cudaSetDevice(device));
+  cudaDeviceProp prop;
+  TALON_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+  if (prop.major < 10) {
+    std::fprintf(stderr, "talon: built for sm_100a, device reports sm_%d%d\n", prop.major, prop.minor);
+    return TALON_ERR_UNSUPPORTED;
+  }
+
+  talon_ctx *c = new (std::nothrow) talon_ctx();
+  if (!c) return TALON_ERR_CUDA;
+  std::memset(c, 0, sizeof(*c));
+  c->p = *p;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->W = (p->budget + 63) / 64;
+  int k = p->cand_topk == 0 ? p->budget - 1 : p->cand_topk;
+  if (k > p->budget - 1) k = p->budget - 1;      // a parent never places more than N-1 children
+  if (k > p->vocab) k = p->vocab;
+  if (k < 1) k = 1;
+  c->k_cap = k;
+  c->k_slots = k <= 32 ? 1 : (k <= 64 ? 2 : 4);
+  c->key_stride = (k + 3) & ~3;
+  c->log_mu = std::log(p->mu);
+  c->exp_grid = c->sm_count * talon::EXP_CTAS_PER_SM;
+  c->rows_cap = p->batch_max * (p->budget - 1);
+  if (c->rows_cap < p->batch_max * p->budget) c->rows_cap = p->batch_max * p->budget;
+  c->items_cap = c->exp_grid + c->rows_cap;
+
+  const size_t nrow = (size_t)p->batch_max * p->budget;
+  bool ok = true;
+  auto alloc = [&](void **ptr, size_t bytes) {
+    if (ok && cudaMalloc(ptr, bytes ? bytes : 16) != cudaSuccess) ok = false;
+  };
+  alloc((void **)&c->d_status, sizeof(int));
+  alloc((void **)&c->d_prefix_len, sizeof(int32_t) * p->batch_max);
+  alloc((void **)&c->d_part_keys, sizeof(unsigned long long) * (size_t)c->items_cap * c->key_stride);
+  alloc((void **)&c->d_part_ms, sizeof(float2) * (size_t)c->items_cap);
+  alloc((void **)&c->d_row_keys, sizeof(unsigned long long) * (size_t)c->rows_cap * c->key_stride);
+  alloc((void **)&c->d_row_lse, sizeof(double) * (size_t)c->rows_cap);
+  alloc((void **)&c->d_row_count, sizeof(unsigned int) * (size_t)c->rows_cap);
+  alloc((void **)&c->d_argmax, sizeof(unsigned long long) * nrow);
+  alloc((void **)&c->d_target_tok, sizeof(int32_t) * nrow);
+  c->attn_o_elems = talon::attention_workspace_elems(c, &c->attn_ml_elems);
+  alloc((void **)&c->d_attn_o, sizeof(float) * c->attn_o_elems);
+  alloc((void **)&c->d_attn_ml, sizeof(float2) * c->attn_ml_elems);
+  if (ok) {
+    ok = cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess &&
+         cudaMemset(c->d_row_count, 0, sizeof(unsigned int) * (size_t)c->rows_cap) == cudaSuccess &&
+         cudaMemset(c->d_argmax, 0, sizeof(unsigned long long) * nrow) == cudaSuccess &&
+         talon::expand_setup(c) == TALON_OK && talon::attention_mma_setup() == TALON_OK;
+  }
+  if (!ok) {
+    std::fprintf(stderr, "talon: context creation failed: %s\n", cudaGetErrorString(cudaGetLastError()));
+    talon_destroy(c);
+    return TALON_ERR_CUDA;
+  }
+  *out_ctx = c;
+  return TALON_OK;
+}
+
+talon_status talon_destroy(talon_ctx *c) {
+  if (!c) return TALON_OK;
+  cudaSetDevice(c->device);
+  cudaFree(c->d_status); cudaFree(c->d_prefix_len); cudaFree(c->d_part_keys); cudaFree(c->d_part_ms);
+  cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_argmax);
+  cudaFree(c->d_target_tok); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
+  free_stage(c->stage);
+  delete c;
+  return TALON_OK;
+}
+
+talon_status talon_reset(talon_ctx *c, const talon_tree *t, const int32_t *root_tok, const int32_t *prefix_len,
+                         int32_t B, void *stream) {
+  if (!c || !tree_complete(t) || !root_tok || !prefix_len) return TALON_ERR_INVALID_ARG;
+  if (B < 1) return TALON_ERR_INVALID_ARG;
+  if (B > c->p.batch_max) return TALON_ERR_CAPACITY;
+  c->B = B;
+  c->layers_run = 0;
+  return talon::launch_reset(c, t, root_tok, prefix_len, B, (cudaStream_t)stream);
+}
+
+talon_status talon_expand_layer(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,
+                                int32_t rows_per_seq, int32_t layout, void *stream) {
+  if (!c || !tree_complete(t) || !logits) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1) return TALON_ERR_INVALID_ARG;                      // no reset yet
+  if (layout != TALON_ROWS_BY_NODE && layout != TALON_ROWS_PACKED) return TALON_ERR_INVALID_ARG;
+  if (row_stride < c->p.vocab || (row_stride & 3) || !aligned16(logits)) return TALON_ERR_INVALID_ARG;
+  if (rows_per_seq < 1 || (layout == TALON_ROWS_BY_NODE && rows_per_seq < c->p.budget)) return TALON_ERR_INVALID_ARG;
+  if (c->layers_run >= c->p.max_depth) return TALON_OK;            // depth stop: nothing to do
+  talon_status s = talon::launch_expand(c, t, logits, row_stride, rows_per_seq, layout, (cudaStream_t)stream);
+  if (s == TALON_OK) c->layers_run += 1;
+  return s;
+}
+
+int32_t talon_layers_run(const talon_ctx *c) { return c ? c->layers_run : -1; }
+
+talon_status talon_build_tree(talon_ctx *c, const talon_tree *t, uint8_t *dense_mask, void *stream) {
+  if (!c || !tree_complete(t)) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1) return TALON_ERR_INVALID_ARG;
+  return talon::launch_build(c, t, dense_mask, (cudaStream_t)stream);
+}
+
+talon_status talon_tree_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *k_prefix,
+                                  const void *v_prefix, const void *k_tree, const void *v_tree,
+                                  const int64_t *kv_start, int64_t kv_stride_t, int64_t kv_stride_h,
+                                  int32_t max_prefix_len, float sm_scale, void *out, void *stream) {
+  if (!c || !tree_complete(t) || !q || !k_tree || !v_tree || !kv_start || !out) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || max_prefix_len < 0) return TALON_ERR_INVALID_ARG;
+  if (max_prefix_len > 0 && (!k_prefix || !v_prefix)) return TALON_ERR_INVALID_ARG;
+  if ((kv_stride_t & 7) || (kv_stride_h & 7) || kv_stride_t < 0 || kv_stride_h < 0) return TALON_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_prefix) || !aligned16(v_prefix) || !aligned16(k_tree) || !aligned16(v_tree) ||
+      !aligned16(out))
+    return TALON_ERR_INVALID_ARG;
+  if (!(sm_scale == sm_scale)) return TALON_ERR_INVALID_ARG;
+  return talon::launch_attention(c, t, q, k_prefix ? k_prefix : k_tree, v_prefix ? v_prefix : v_tree, k_tree,
+                                 v_tree, kv_start, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out,
+                                 (cudaStream_t)stream);
+}
+
+talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                          int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                          void *stream) {
+  if (!c || !tree_complete(t) || !target_logits || !accept_len || !accept_nodes || !bonus_tok)
+    return TALON_ERR_INVALID_ARG;
+  if (c->B < 1) return TALON_ERR_INVALID_ARG;
+  if (row_stride < c->p.vocab || (row_stride & 3) || !aligned16(target_logits)) return TALON_ERR_INVALID_ARG;
+  return talon::launch_accept(c, t, target_logits, row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
+                              (cudaStream_t)stream);
+}
+
+talon_status talon_poll_status(talon_ctx *c, void *stream) {
+  if (!c) return TALON_ERR_INVALID_ARG;
+  int word = 0;
+  TALON_CUDA_OK(cudaMemcpyAsync(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  TALON_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  if (word & talon::STATUS_TIMEOUT) return TALON_ERR_TIMEOUT;
+  if (word & talon::STATUS_CAPACITY) return TALON_ERR_CAPACITY;
+  if (word & talon::STATUS_NONFINITE) return TALON_ERR_NONFINITE;
+  return TALON_OK;
+}
+
+int64_t talon_launch_count(const talon_ctx *c) { return c ? c->launches : -1; }
+
+talon_status talon_step_host(talon_ctx *c, int32_t B, const int32_t *root_tok, const int32_t *prefix_len,
+                             const float *draft_logits, const float *target_logits, const void *q,
+                             const void *k_prefix, const void *v_prefix, const void *k_tree, const void *v_tree,
+                             float sm_scale, void *out_attn, int32_t *n_nodes, int32_t *token, int32_t *parent,
+                             int32_t *depth, int32_t *position, int32_t *accept_len, int32_t *accept_nodes,
+                             int32_t *bonus_tok, void *stream) {
+  if (!c || !root_tok || !prefix_len || !draft_logits || !target_logits || !q || !k_tree || !v_tree ||
+      !accept_len || !accept_nodes || !bonus_tok)
+    return TALON_ERR_INVALID_ARG;
+  if (B < 1) return TALON_ERR_INVALID_ARG;
+  if (B > c->p.batch_max) return TALON_ERR_CAPACITY;
+  cudaStream_t st = (cudaStream_t)stream;
+  const talon_params &p = c->p;
+  const size_t N = p.budget, V = p.vocab, Dh = p.head_dim;
+  if (V & 3) return TALON_ERR_UNSUPPORTED;        // dense [B,N,V] rows must stay 16-byte aligned
+
+  int64_t tokens = 0;
+  int max_len = 0;
+  for (int b = 0; b < B; ++b) {
+    if (prefix_len[b] < 0) return TALON_ERR_INVALID_ARG;
+    tokens += prefix_len[b];
+    if (prefix_len[b] > max_len) max_len = prefix_len[b];
+  }
+  if (tokens > 0 && (!k_prefix || !v_prefix)) return TALON_ERR_INVALID_ARG;
+  TALON_CUDA_OK(cudaSetDevice(c->device));
+
+  HostStage *s = c->stage;
+  if (!s || s->prefix_tokens < tokens) {
+    TALON_CUDA_OK(cudaStreamSynchronize(st));
+    free_stage(s);
+    c->stage = nullptr;
+    s = new (std::nothrow) HostStage();
+    if (!s) return TALON_ERR_CUDA;
+    c->stage = s;
+    const size_t bm = p.batch_max, W = c->W;
+    s->batch = p.batch_max;
+    s->prefix_tokens = tokens > 0 ? tokens : 1;
+    TALON_CUDA_OK(cudaMalloc((void **)&s->draft, bm * N * V * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->target, bm * N * V * 4));
+    TALON_CUDA_OK(cudaMalloc(&s->q, bm * N * p.n_q_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc(&s->out, bm * N * p.n_q_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc(&s->kp, (size_t)s->prefix_tokens * p.n_kv_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc(&s->vp, (size_t)s->prefix_tokens * p.n_kv_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc(&s->kt, bm * N * p.n_kv_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc(&s->vt, bm * N * p.n_kv_heads * Dh * 2));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->root, bm * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->plen, bm * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->kv_start, bm * 8));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.n_nodes, bm * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.token, bm * N * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.parent, bm * N * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.depth, bm * N * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.position, bm * N * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.layer_off, bm * (p.max_depth + 2) * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.score, bm * N * 8));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->tree.mask, bm * N * W * 8));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->accept_len, bm * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->accept_nodes, bm * (p.max_depth + 1) * 4));
+    TALON_CUDA_OK(cudaMalloc((void **)&s->bonus, bm * 4));
+    TALON_CUDA_OK(cudaMallocHost((void **)&s->h_kv_start, bm * 8));
+  }
+
+  {
+    int64_t run = 0;
+    for (int b = 0; b < B; ++b) { s->h_kv_start[b] = run; run += prefix_len[b]; }
+  }
+  const size_t rows = (size_t)B * N;
+  const size_t kvrow = (size_t)p.n_kv_heads * Dh * 2;
+#define H2D(dst, src, bytes) TALON_CUDA_OK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st))
+#define D2H(dst, src, bytes) TALON_CUDA_OK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st))
+  H2D(s->root, root_tok, (size_t)B * 4);
+  H2D(s->plen, prefix_len, (size_t)B * 4);
+  H2D(s->kv_start, s->h_kv_start, (size_t)B * 8);
+  H2D(s->draft, draft_logits, rows * V * 4);
+  H2D(s->target, target_logits, rows * V * 4);
+  H2D(s->q, q, rows * p.n_q_heads * Dh * 2);
+  if (tokens > 0) {
+    H2D(s->kp, k_prefix, (size_t)tokens * kvrow);
+    H2D(s->vp, v_prefix, (size_t)tokens * kvrow);
+  }
+  H2D(s->kt, k_tree, rows * kvrow);
+  H2D(s->vt, v_tree, rows * kvrow);
+
+  talon_status r = talon_reset(c, &s->tree, s->root, s->plen, B, stream);
+  for (int d = 0; r == TALON_OK && d < p.max_depth; ++d)
+    r = talon_expand_layer(c, &s->tree, s->draft, (int64_t)V, (int32_t)N, TALON_ROWS_BY_NODE, stream);
+  if (r == TALON_OK) r = talon_build_tree(c, &s->tree, nullptr, stream);
+  if (r == TALON_OK)
+    r = talon_tree_attention(c, &s->tree, s->q, s->kp, s->vp, s->kt, s->vt, s->kv_start,
+                             (int64_t)p.n_kv_heads * Dh, (int64_t)Dh, max_len, sm_scale, s->out, stream);
+  if (r == TALON_OK)
+    r = talon_accept(c, &s->tree, s->target, (int64_t)V, nullptr, s->accept_len, s->accept_nodes, s->bonus, stream);
+  if (r != TALON_OK) return r;
+
+  if (out_attn) D2H(out_attn, s->out, rows * p.n_q_heads * Dh * 2);
+  if (n_nodes) D2H(n_nodes, s->tree.n_nodes, (size_t)B * 4);
+  if (token) D2H(token, s->tree.token, rows * 4);
+  if (parent) D2H(parent, s->tree.parent, rows * 4);
+  if (depth) D2H(depth, s->tree.depth, rows * 4);
+  if (position) D2H(position, s->tree.position, rows * 4);
+  D2H(accept_len, s->accept_len, (size_t)B * 4);
+  D2H(accept_nodes, s->accept_nodes, (size_t)B * (p.max_depth + 1) * 4);
+  D2H(bonus_tok, s->bonus, (size_t)B * 4);
+#undef H2D
+#undef D2H
+  return talon_poll_status(c, stream);
+}
+
+}  // extern "C"

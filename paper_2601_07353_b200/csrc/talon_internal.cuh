@@ -1,0 +1,128 @@
+// Internal declarations shared by the translation units of libtalon (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "talon.h"
+
+namespace talon {
+
+// ---- device status bits (ctx->d_status) -----------------------------------------------
+constexpr int STATUS_NONFINITE = 1;
+constexpr int STATUS_TIMEOUT = 2;
+constexpr int STATUS_CAPACITY = 4;
+
+// ---- expansion geometry -----------------------------------------------------------------
+constexpr int EXP_THREADS = 256;           // threads per CTA of the row-streaming kernels
+constexpr int EXP_WARPS = EXP_THREADS / 32;
+constexpr int EXP_VEC = 4;                 // floats per 128-bit load
+constexpr int EXP_UNROLL = 4;              // 128-bit loads in flight per thread
+constexpr int EXP_TILE = EXP_THREADS * EXP_VEC * EXP_UNROLL;   // 4096 elements per CTA step
+constexpr int EXP_CHUNK_ALIGN = EXP_THREADS * EXP_VEC;         // chunk boundaries: 1024 elements
+constexpr int EXP_MAX_SPLITS = 32;         // a row is cut into at most this many chunks
+constexpr int EXP_CTAS_PER_SM = 4;
+constexpr int MAX_BUDGET = 128;
+constexpr int MAX_BATCH = 1024;
+constexpr int SEL_THREADS = 512;
+
+// Order-preserving map fp32 -> u32 (larger float <=> larger integer; -inf > 0).
+__host__ __device__ inline uint32_t f32_ord(float f) {
+#ifdef __CUDA_ARCH__
+  uint32_t b = __float_as_uint(f);
+#else
+  union { float f; uint32_t u; } c; c.f = f; uint32_t b = c.u;
+#endif
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__host__ __device__ inline float f32_unord(uint32_t o) {
+  uint32_t b = (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o;
+#ifdef __CUDA_ARCH__
+  return __uint_as_float(b);
+#else
+  union { float f; uint32_t u; } c; c.u = b; return c.f;
+#endif
+}
+// A candidate key: larger key = larger logit, then lower token id.  Key 0 means "empty".
+__host__ __device__ inline uint64_t cand_key(float logit, uint32_t tok) {
+  return ((uint64_t)f32_ord(logit) << 32) | (uint64_t)(0xFFFFFFFFu - tok);
+}
+__host__ __device__ inline float key_logit(uint64_t k) { return f32_unord((uint32_t)(k >> 32)); }
+__host__ __device__ inline uint32_t key_tok(uint64_t k) { return 0xFFFFFFFFu - (uint32_t)k; }
+
+// How one expansion layer is cut into work items.  Computed identically (from device data)
+// by every CTA of the streaming kernel and by the selection kernel.
+struct LayerGeom {
+  int total_rows;   // frontier rows over all sequences
+  int splits;       // chunks per row
+  int chunk_len;    // elements per chunk (multiple of EXP_CHUNK_ALIGN)
+};
+
+__host__ __device__ inline LayerGeom make_geom(int total_rows, int vocab, int target_items) {
+  LayerGeom g;
+  g.total_rows = total_rows;
+  int want = total_rows > 0 ? (target_items + total_rows - 1) / total_rows : 1;
+  if (want < 1) want = 1;
+  if (want > EXP_MAX_SPLITS) want = EXP_MAX_SPLITS;
+  int len = (vocab + want - 1) / want;
+  len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
+  g.chunk_len = len;
+  g.splits = (vocab + len - 1) / len;
+  return g;
+}
+
+}  // namespace talon
+
+// The context: parameters, host-side counters, and the device workspace.
+struct talon_ctx {
+  talon_params p;
+  int device;
+  int sm_count;
+  int W;                  // mask words per node
+  int k_cap;              // per-parent candidate cap actually used (cand_topk or N-1)
+  int k_slots;            // ceil(k_cap / 32): list registers per lane
+  int key_stride;         // keys stored per row / per item (k_cap rounded up to 4)
+  int B;                  // batch of the current reset
+  int layers_run;         // expand calls since reset
+  int64_t launches;
+  double log_mu;
+
+  int *d_status;
+  int32_t *d_prefix_len;          // [batch_max]
+  // expansion workspace
+  int exp_grid;                   // CTAs of the streaming kernel at full width
+  int rows_cap;                   // batch_max * (N-1)
+  int items_cap;                  // exp_grid + rows_cap
+  unsigned long long *d_part_keys;   // [items_cap, key_stride]  per-chunk top-k
+  float2 *d_part_ms;                 // [items_cap]              per-chunk (max, sum exp)
+  unsigned long long *d_row_keys;    // [rows_cap, key_stride]   per-row top-k
+  double *d_row_lse;                 // [rows_cap]               per-row log-sum-exp
+  unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
+  // verification workspace
+  unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
+  int32_t *d_target_tok;             // [batch_max * N]
+  float *d_attn_o;                   // split-KV partial outputs
+  float2 *d_attn_ml;                 // split-KV partial (max, sum)
+  size_t attn_o_elems, attn_ml_elems;
+  // host-step staging (allocated on first use)
+  struct HostStage *stage;
+};
+
+namespace talon {
+
+// launchers implemented in the .cu files (all asynchronous on `st`)
+talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root_tok,
+                          const int32_t *prefix_len, int B, cudaStream_t st);
+talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logits,
+                           int64_t row_stride, int rows_per_seq, int layout, cudaStream_t st);
+talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cudaStream_t st);
+talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp,
+                              const void *vp, const void *kt, const void *vt,
+                              const int64_t *kv_start, int64_t stride_t, int64_t stride_h,
+                              int max_prefix_len, float sm_scale, void *out, cudaStream_t st);
+talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
+                           int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
+                           int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st);
+size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems);
+
+}  // namespace talon

@@ -1,0 +1,191 @@
+"""Thin ctypes binding over ``libtalon.so`` (the C ABI declared in ``include/talon.h``).
+
+Only argument marshalling happens here: torch supplies device memory and streams, every step
+of the path runs in the library's CUDA kernels.  There is no CPU fallback: if the library has
+not been built (``python -m paper_2601_07353_b200.build``) importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtalon.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build the CUDA library first with "
+        "`python -m paper_2601_07353_b200.build` (needs nvcc); there is no CPU fallback")
+_lib = C.CDLL(_LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_UNSUPPORTED = range(7)
+ROWS_BY_NODE, ROWS_PACKED = 0, 1
+
+
+class TalonParams(C.Structure):
+    _fields_ = [("batch_max", C.c_int32), ("vocab", C.c_int32), ("budget", C.c_int32),
+                ("root_topk", C.c_int32), ("cand_topk", C.c_int32), ("max_depth", C.c_int32),
+                ("init_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("mu", C.c_double)]
+
+
+class TalonTreeStruct(C.Structure):
+    _fields_ = [("n_nodes", C.c_void_p), ("token", C.c_void_p), ("parent", C.c_void_p),
+                ("depth", C.c_void_p), ("position", C.c_void_p), ("layer_off", C.c_void_p),
+                ("score", C.c_void_p), ("mask", C.c_void_p)]
+
+
+_vp, _i32, _i64, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+_TP = C.POINTER(TalonTreeStruct)
+_lib.talon_create.argtypes = [C.POINTER(_vp), C.POINTER(TalonParams), C.c_int]
+_lib.talon_destroy.argtypes = [_vp]
+_lib.talon_reset.argtypes = [_vp, _TP, _vp, _vp, _i32, _vp]
+_lib.talon_expand_layer.argtypes = [_vp, _TP, _vp, _i64, _i32, _i32, _vp]
+_lib.talon_layers_run.argtypes = [_vp]
+_lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
+_lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp]
+_lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.talon_poll_status.argtypes = [_vp, _vp]
+_lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
+_lib.talon_launch_count.argtypes = [_vp]
+_lib.talon_launch_count.restype = C.c_int64
+_lib.talon_status_string.argtypes = [C.c_int]
+_lib.talon_status_string.restype = C.c_char_p
+for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
+           "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host"):
+    getattr(_lib, _n).restype = C.c_int
+
+EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
+            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
+            "talon_step_host", "talon_launch_count", "talon_status_string"]
+
+
+class TalonError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_lib.talon_status_string(code).decode()} ({code})")
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise TalonError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+@dataclass
+class Tree:
+    """Caller-owned device arrays of the draft tree (``talon_tree`` in the header)."""
+    n_nodes: torch.Tensor
+    token: torch.Tensor
+    parent: torch.Tensor
+    depth: torch.Tensor
+    position: torch.Tensor
+    layer_off: torch.Tensor
+    score: torch.Tensor
+    mask: torch.Tensor
+
+    def struct(self) -> TalonTreeStruct:
+        return TalonTreeStruct(*(t.data_ptr() for t in (self.n_nodes, self.token, self.parent, self.depth,
+                                                          self.position, self.layer_off, self.score, self.mask)))
+
+
+class Talon:
+    """One library context (``talon_ctx``) on one CUDA device; methods mirror the C calls."""
+
+    def __init__(self, *, batch_max, vocab, budget, root_topk, cand_topk, max_depth, n_q_heads, n_kv_heads,
+                 head_dim=128, mu=0.03, init_layers=1, device=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("talon needs a CUDA device; there is no CPU path")
+        self.device = torch.device("cuda", device)
+        self.params = TalonParams(batch_max, vocab, budget, root_topk, cand_topk, max_depth, init_layers,
+                                  n_q_heads, n_kv_heads, head_dim, mu)
+        self._ctx = C.c_void_p()
+        _check(_lib.talon_create(C.byref(self._ctx), C.byref(self.params), device), "talon_create")
+        self.N, self.V, self.W = budget, vocab, (budget + 63) // 64
+
+    def close(self):
+        if self._ctx:
+            _lib.talon_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def alloc_tree(self, B: int) -> Tree:
+        d, N = self.device, self.N
+        i32 = dict(dtype=torch.int32, device=d)
+        return Tree(torch.zeros(B, **i32), torch.zeros(B, N, **i32), torch.zeros(B, N, **i32),
+                    torch.zeros(B, N, **i32), torch.zeros(B, N, **i32),
+                    torch.zeros(B, self.params.max_depth + 2, **i32),
+                    torch.zeros(B, N, dtype=torch.float64, device=d),
+                    torch.zeros(B, N, self.W, dtype=torch.int64, device=d))
+
+    def reset(self, tree: Tree, root_tok: torch.Tensor, prefix_len: torch.Tensor):
+        B = root_tok.shape[0]
+        ts = tree.struct()
+        _check(_lib.talon_reset(self._ctx, C.byref(ts), _ptr(root_tok), _ptr(prefix_len), B,
+                                _stream(self.device)), "talon_reset")
+
+    def expand_layer(self, tree: Tree, logits: torch.Tensor, rows_per_seq: Optional[int] = None,
+                     layout: int = ROWS_BY_NODE, row_stride: Optional[int] = None):
+        ts = tree.struct()
+        if row_stride is None:
+            row_stride = logits.stride(-2)
+        if rows_per_seq is None:
+            rows_per_seq = logits.shape[-2]
+        _check(_lib.talon_expand_layer(self._ctx, C.byref(ts), _ptr(logits), row_stride, rows_per_seq, layout,
+                                       _stream(self.device)), "talon_expand_layer")
+
+    def layers_run(self) -> int:
+        return _lib.talon_layers_run(self._ctx)
+
+    def build_tree(self, tree: Tree, dense_mask: Optional[torch.Tensor] = None):
+        ts = tree.struct()
+        _check(_lib.talon_build_tree(self._ctx, C.byref(ts), _ptr(dense_mask), _stream(self.device)),
+               "talon_build_tree")
+
+    def tree_attention(self, tree: Tree, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_stride_t,
+                       kv_stride_h, max_prefix_len, sm_scale, out):
+        ts = tree.struct()
+        _check(_lib.talon_tree_attention(self._ctx, C.byref(ts), _ptr(q), _ptr(k_prefix), _ptr(v_prefix),
+                                         _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_stride_t, kv_stride_h,
+                                         max_prefix_len, sm_scale, _ptr(out), _stream(self.device)),
+               "talon_tree_attention")
+
+    def accept(self, tree: Tree, target_logits, accept_len, accept_nodes, bonus_tok, target_tok=None,
+               row_stride: Optional[int] = None):
+        ts = tree.struct()
+        if row_stride is None:
+            row_stride = target_logits.stride(-2)
+        _check(_lib.talon_accept(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, _ptr(target_tok),
+                                 _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok), _stream(self.device)),
+               "talon_accept")
+
+    def poll_status(self) -> int:
+        return _lib.talon_poll_status(self._ctx, _stream(self.device))
+
+    def launch_count(self) -> int:
+        return _lib.talon_launch_count(self._ctx)
+
+    def step_host(self, root_tok, prefix_len, draft_logits, target_logits, q, k_prefix, v_prefix, k_tree, v_tree,
+                  sm_scale, out_attn, n_nodes, token, parent, depth, position, accept_len, accept_nodes,
+                  bonus_tok) -> int:
+        """All arguments are HOST tensors (pinned for asynchronous copies).  Returns the status."""
+        B = root_tok.shape[0]
+        return _lib.talon_step_host(self._ctx, B, _ptr(root_tok), _ptr(prefix_len), _ptr(draft_logits),
+                                    _ptr(target_logits), _ptr(q), _ptr(k_prefix), _ptr(v_prefix), _ptr(k_tree),
+                                    _ptr(v_tree), sm_scale, _ptr(out_attn), _ptr(n_nodes), _ptr(token),
+                                    _ptr(parent), _ptr(depth), _ptr(position), _ptr(accept_len),
+                                    _ptr(accept_nodes), _ptr(bonus_tok), _stream(self.device))
