@@ -188,8 +188,55 @@ talon_status talon_step_host(talon_ctx *ctx, int32_t B, const int32_t *root_tok,
                              int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
                              void *stream);
 
+/* Device buffers in, device results out: the same whole step as talon_step_host (Algorithm 2
+ * until the budget or D_max is reached, then Appendix B's verification) as one call, so that a
+ * caller pays for one library entry instead of D_max + 4.  Every pointer is DEVICE memory with
+ * the layout of the call it is handed to: talon_reset (root_tok, prefix_len), talon_expand_layer
+ * with rows BY_NODE (draft_logits, draft_row_stride, N rows per sequence), talon_tree_attention
+ * (q .. out), talon_accept (target_logits .. bonus_tok; target_tok may be null).
+ * n_layers  expansion layers to enqueue, 0..D_max (layers after the tree is full cost one
+ *           frontier check each and read no logits)
+ * Enqueues only; no synchronisation. */
+talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const int32_t *root_tok,
+                        const int32_t *prefix_len, const float *draft_logits,
+                        int64_t draft_row_stride, int32_t n_layers, const void *q,
+                        const void *k_prefix, const void *v_prefix, const void *k_tree,
+                        const void *v_tree, const int64_t *kv_start, int64_t kv_stride_t,
+                        int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
+                        int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                        void *stream);
+
 /* Number of kernels the library has launched through this context since creation. */
 int64_t talon_launch_count(const talon_ctx *ctx);
+
+/* Kernel families of the library, for talon_timing_read. */
+enum {
+  TALON_K_RESET = 0,        /* tree initialisation (Algorithm 2, lines 1-2)                  */
+  TALON_K_EXPAND_ROWS = 1,  /* softmax normaliser + per-parent top-k over the logit rows    */
+  TALON_K_SELECT = 2,       /* Top-K / gate / budget truncation / append                    */
+  TALON_K_BUILD = 3,        /* positions and sentinels                                      */
+  TALON_K_ATTENTION = 4,    /* tree attention                                               */
+  TALON_K_COMBINE = 5,      /* merge of split-KV partials                                   */
+  TALON_K_ARGMAX = 6,       /* target argmax                                                */
+  TALON_K_WALK = 7,         /* greedy accept walk                                           */
+  TALON_N_KERNELS = 8
+};
+
+/* Per-kernel device timing.  With max_launches > 0 the context creates that many pairs of
+ * CUDA events (an allocation; synchronises the device) and from then on brackets every launch
+ * of the kernel families in kernel_mask (bit k = family k; 0 = all) with a pair recorded on the
+ * launching stream, until the pairs run out.  max_launches = 0 switches timing off and destroys
+ * the events.  Do not capture a stream into a CUDA graph while timing is on. */
+talon_status talon_timing_enable(talon_ctx *ctx, int32_t max_launches, uint32_t kernel_mask);
+
+/* Synchronises `stream`, adds up the elapsed time of the bracketed launches per kernel family
+ * since the last read, and makes all pairs available again.
+ * ms        host [TALON_N_KERNELS] summed milliseconds
+ * launches  host [TALON_N_KERNELS] number of launches that were timed */
+talon_status talon_timing_read(talon_ctx *ctx, void *stream, double *ms, int64_t *launches);
+
+const char *talon_kernel_name(int32_t kernel);
 
 const char *talon_status_string(talon_status s);
 

@@ -144,7 +144,10 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   long long items = (long long)rows * g.splits;
   int grid = c->exp_grid;
   if (items < grid) grid = (int)items;
-  target_argmax_kernel<<<grid, EXP_THREADS, 0, st>>>(aa);
+  {
+    LaunchTimer lt(c, TALON_K_ARGMAX, st);
+    target_argmax_kernel<<<grid, EXP_THREADS, 0, st>>>(aa);
+  }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
 
   WalkArgs wa;
@@ -153,7 +156,10 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   wa.best = c->d_argmax; wa.target_tok = target_tok ? target_tok : c->d_target_tok;
   wa.accept_len = accept_len; wa.accept_nodes = accept_nodes; wa.bonus_tok = bonus_tok;
   const int warps_per_block = 4;
-  accept_walk_kernel<<<(c->B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(wa);
+  {
+    LaunchTimer lt(c, TALON_K_WALK, st);
+    accept_walk_kernel<<<(c->B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(wa);
+  }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 2;
   return TALON_OK;

@@ -152,6 +152,7 @@ talon_status talon_destroy(talon_ctx *c) {
   cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_argmax);
   cudaFree(c->d_target_tok); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
+  talon_timing_enable(c, 0, 0u);
   delete c;
   return TALON_OK;
 }
@@ -227,6 +228,78 @@ talon_status talon_poll_status(talon_ctx *c, void *stream) {
 }
 
 int64_t talon_launch_count(const talon_ctx *c) { return c ? c->launches : -1; }
+
+const char *talon_kernel_name(int32_t k) {
+  switch (k) {
+    case TALON_K_RESET: return "reset";
+    case TALON_K_EXPAND_ROWS: return "expand_rows";
+    case TALON_K_SELECT: return "select_layer";
+    case TALON_K_BUILD: return "build_tree";
+    case TALON_K_ATTENTION: return "tree_attention";
+    case TALON_K_COMBINE: return "attention_combine";
+    case TALON_K_ARGMAX: return "target_argmax";
+    case TALON_K_WALK: return "accept_walk";
+  }
+  return "unknown";
+}
+
+talon_status talon_timing_enable(talon_ctx *c, int32_t max_launches, uint32_t kernel_mask) {
+  if (!c || max_launches < 0) return TALON_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  if (c->ev) {
+    cudaDeviceSynchronize();
+    for (int i = 0; i < 2 * c->ev_cap; ++i) cudaEventDestroy(c->ev[i]);
+    delete[] c->ev;
+    delete[] c->ev_kernel;
+    c->ev = nullptr; c->ev_kernel = nullptr; c->ev_cap = c->ev_used = 0;
+  }
+  if (max_launches == 0) return TALON_OK;
+  c->ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
+  c->ev_kernel = new (std::nothrow) int[max_launches];
+  if (!c->ev || !c->ev_kernel) return TALON_ERR_CUDA;
+  for (int i = 0; i < 2 * max_launches; ++i) TALON_CUDA_OK(cudaEventCreate(&c->ev[i]));
+  c->ev_cap = max_launches;
+  c->ev_used = 0;
+  c->ev_mask = kernel_mask ? kernel_mask : 0xFFFFFFFFu;
+  return TALON_OK;
+}
+
+talon_status talon_timing_read(talon_ctx *c, void *stream, double *ms, int64_t *launches) {
+  if (!c || !ms || !launches) return TALON_ERR_INVALID_ARG;
+  for (int k = 0; k < TALON_N_KERNELS; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  if (!c->ev) return TALON_OK;
+  TALON_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  for (int i = 0; i < c->ev_used; ++i) {
+    float t = 0.f;
+    TALON_CUDA_OK(cudaEventElapsedTime(&t, c->ev[2 * i], c->ev[2 * i + 1]));
+    const int k = c->ev_kernel[i];
+    if (k >= 0 && k < TALON_N_KERNELS) { ms[k] += t; launches[k] += 1; }
+  }
+  c->ev_used = 0;
+  return TALON_OK;
+}
+
+talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
+                        const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
+                        int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
+                        const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_stride_t,
+                        int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
+                        int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok, void *stream) {
+  if (!c) return TALON_ERR_INVALID_ARG;
+  if (n_layers < 0 || n_layers > c->p.max_depth) return TALON_ERR_INVALID_ARG;
+  talon_status r = talon_reset(c, t, root_tok, prefix_len, B, stream);
+  for (int d = 0; r == TALON_OK && d < n_layers; ++d)
+    r = talon_expand_layer(c, t, draft_logits, draft_row_stride, c->p.budget, TALON_ROWS_BY_NODE, stream);
+  if (r == TALON_OK) r = talon_build_tree(c, t, nullptr, stream);
+  if (r == TALON_OK)
+    r = talon_tree_attention(c, t, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_stride_t, kv_stride_h,
+                             max_prefix_len, sm_scale, out, stream);
+  if (r == TALON_OK)
+    r = talon_accept(c, t, target_logits, target_row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
+                     stream);
+  return r;
+}
 
 talon_status talon_step_host(talon_ctx *c, int32_t B, const int32_t *root_tok, const int32_t *prefix_len,
                              const float *draft_logits, const float *target_logits, const void *q,

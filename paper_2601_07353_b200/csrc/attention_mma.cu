@@ -369,12 +369,16 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
   a.splits = splits;
 
   dim3 grid(a.m_blocks, splits, c->B * a.Hkv);
-  tree_attention_mma_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(a);
+  {
+    LaunchTimer lt(c, TALON_K_ATTENTION, st);
+    tree_attention_mma_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(a);
+  }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;
   if (splits > 1) {
     const int64_t rows = (int64_t)c->B * a.Hkv * a.g * a.N;
     const int wpb = 8;
+    LaunchTimer lt(c, TALON_K_COMBINE, st);
     attention_combine_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(a);
     if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
     c->launches += 1;

@@ -669,6 +669,7 @@ talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root
   int blocks = (c->rows_cap + threads - 1) / threads;
   if (blocks > 64) blocks = 64;
   if (blocks < 1) blocks = 1;
+  LaunchTimer lt(c, TALON_K_RESET, st);
   reset_kernel<<<blocks, threads, 0, st>>>(*t, root_tok, prefix_len, c->d_prefix_len, B, c->p.budget, c->W,
                                            c->p.max_depth + 2, c->d_status, c->d_row_count, c->rows_cap);
   c->launches += 1;
@@ -692,10 +693,13 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
   ea.part_keys = c->d_part_keys; ea.part_ms = c->d_part_ms; ea.row_keys = c->d_row_keys;
   ea.row_lse = c->d_row_lse; ea.row_count = c->d_row_count; ea.status = c->d_status;
   const size_t lists_bytes = (size_t)EXP_MAX_SPLITS * 32 * c->k_slots * sizeof(unsigned long long);
-  switch (c->k_slots) {
-    case 1: expand_rows_kernel<1><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
-    case 2: expand_rows_kernel<2><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
-    default: expand_rows_kernel<4><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
+  {
+    LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
+    switch (c->k_slots) {
+      case 1: expand_rows_kernel<1><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
+      case 2: expand_rows_kernel<2><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
+      default: expand_rows_kernel<4><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
+    }
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
 
@@ -706,13 +710,17 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
   sa.root_topk = c->p.root_topk; sa.init_layers = c->p.init_layers; sa.log_mu = c->log_mu;
   sa.row_keys = c->d_row_keys; sa.row_lse = c->d_row_lse; sa.status = c->d_status;
   sa.pool_cap = pool_capacity(c);
-  select_layer_kernel<<<c->B, SEL_THREADS, select_smem_bytes(sa.pool_cap), st>>>(sa);
+  {
+    LaunchTimer lt(c, TALON_K_SELECT, st);
+    select_layer_kernel<<<c->B, SEL_THREADS, select_smem_bytes(sa.pool_cap), st>>>(sa);
+  }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 2;
   return TALON_OK;
 }
 
 talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cudaStream_t st) {
+  LaunchTimer lt(c, TALON_K_BUILD, st);
   build_tree_kernel<<<c->B, 128, 0, st>>>(*t, c->d_prefix_len, dense, c->B, c->p.budget, c->W,
                                           c->p.max_depth + 2, c->layers_run);
   c->launches += 1;

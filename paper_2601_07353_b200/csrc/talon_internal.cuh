@@ -106,9 +106,32 @@ struct talon_ctx {
   size_t attn_o_elems, attn_ml_elems;
   // host-step staging (allocated on first use)
   struct HostStage *stage;
+  // per-kernel timing (off unless talon_timing_enable was called)
+  cudaEvent_t *ev;                   // [2 * ev_cap] start/stop pairs
+  int *ev_kernel;                    // [ev_cap] kernel id of each pair
+  int ev_cap, ev_used;
+  unsigned ev_mask;                  // kernel families that are timed
 };
 
 namespace talon {
+
+// Brackets one kernel launch with a pair of CUDA events on the launching stream when timing
+// is on; does nothing otherwise.  Pairs beyond the capacity are silently not timed.
+struct LaunchTimer {
+  talon_ctx *c;
+  cudaStream_t st;
+  int slot;
+  LaunchTimer(talon_ctx *ctx, int kernel, cudaStream_t stream) : c(ctx), st(stream), slot(-1) {
+    if (c->ev && ((c->ev_mask >> kernel) & 1u) && c->ev_used < c->ev_cap) {
+      slot = c->ev_used++;
+      c->ev_kernel[slot] = kernel;
+      cudaEventRecord(c->ev[2 * slot], st);
+    }
+  }
+  ~LaunchTimer() {
+    if (slot >= 0) cudaEventRecord(c->ev[2 * slot + 1], st);
+  }
+};
 
 // launchers implemented in the .cu files (all asynchronous on `st`)
 talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root_tok,

@@ -49,17 +49,27 @@ _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_poll_status.argtypes = [_vp, _vp]
 _lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
+_lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i32, _f32, _vp,
+                            _vp, _i64] + [_vp] * 5)
+_lib.talon_timing_enable.argtypes = [_vp, _i32, C.c_uint32]
+_lib.talon_timing_read.argtypes = [_vp, _vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+_lib.talon_kernel_name.argtypes = [_i32]
+_lib.talon_kernel_name.restype = C.c_char_p
 _lib.talon_launch_count.argtypes = [_vp]
 _lib.talon_launch_count.restype = C.c_int64
 _lib.talon_status_string.argtypes = [C.c_int]
 _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
-           "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host"):
+           "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
+           "talon_step", "talon_timing_enable", "talon_timing_read"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
             "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
-            "talon_step_host", "talon_launch_count", "talon_status_string"]
+            "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_kernel_name",
+            "talon_launch_count", "talon_status_string"]
+N_KERNELS = 8
+KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
 
 
 class TalonError(RuntimeError):
@@ -178,6 +188,32 @@ class Talon:
 
     def launch_count(self) -> int:
         return _lib.talon_launch_count(self._ctx)
+
+    def step(self, tree: Tree, root_tok, prefix_len, draft_logits, n_layers, q, k_prefix, v_prefix, k_tree, v_tree,
+             kv_start, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out, target_logits, target_tok,
+             accept_len, accept_nodes, bonus_tok):
+        """``talon_step``: the whole draft-and-verify step on device-resident inputs, one library call."""
+        ts = tree.struct()
+        _check(_lib.talon_step(self._ctx, C.byref(ts), root_tok.shape[0], _ptr(root_tok), _ptr(prefix_len),
+                               _ptr(draft_logits), draft_logits.stride(-2), n_layers, _ptr(q), _ptr(k_prefix),
+                               _ptr(v_prefix), _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_stride_t, kv_stride_h,
+                               max_prefix_len, sm_scale, _ptr(out), _ptr(target_logits), target_logits.stride(-2),
+                               _ptr(target_tok), _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok),
+                               _stream(self.device)), "talon_step")
+
+    def timing_enable(self, max_launches: int, kernels=None):
+        """Bracket launches with CUDA events; ``kernels`` = names to time (None: all); 0 switches off."""
+        mask = 0
+        for k in kernels or ():
+            mask |= 1 << KERNEL_NAMES.index(k)
+        _check(_lib.talon_timing_enable(self._ctx, max_launches, mask), "talon_timing_enable")
+
+    def timing_read(self):
+        """Returns {kernel name: (summed ms, launches)} since the last read (synchronises the stream)."""
+        ms = (C.c_double * N_KERNELS)()
+        n = (C.c_int64 * N_KERNELS)()
+        _check(_lib.talon_timing_read(self._ctx, _stream(self.device), ms, n), "talon_timing_read")
+        return {KERNEL_NAMES[i]: (ms[i], n[i]) for i in range(N_KERNELS)}
 
     def step_host(self, root_tok, prefix_len, draft_logits, target_logits, q, k_prefix, v_prefix, k_tree, v_tree,
                   sm_scale, out_attn, n_nodes, token, parent, depth, position, accept_len, accept_nodes,
