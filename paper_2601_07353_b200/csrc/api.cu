@@ -125,6 +125,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
   alloc((void **)&c->d_row_keys, sizeof(unsigned long long) * (size_t)c->rows_cap * c->key_stride);
   alloc((void **)&c->d_row_lse, sizeof(double) * (size_t)c->rows_cap);
   alloc((void **)&c->d_row_count, sizeof(unsigned int) * (size_t)c->rows_cap);
+  alloc((void **)&c->d_seq_count, sizeof(unsigned int) * (size_t)p->batch_max);
   alloc((void **)&c->d_argmax, sizeof(unsigned long long) * nrow);
   alloc((void **)&c->d_target_tok, sizeof(int32_t) * nrow);
   c->attn_o_elems = talon::attention_workspace_elems(c, &c->attn_ml_elems);
@@ -134,7 +135,10 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     ok = cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess &&
          cudaMemset(c->d_row_count, 0, sizeof(unsigned int) * (size_t)c->rows_cap) == cudaSuccess &&
          cudaMemset(c->d_argmax, 0, sizeof(unsigned long long) * nrow) == cudaSuccess &&
-         talon::expand_setup(c) == TALON_OK && talon::attention_mma_setup() == TALON_OK;
+         cudaMemset(c->d_seq_count, 0, sizeof(unsigned int) * (size_t)p->batch_max) == cudaSuccess &&
+         cudaMemset(c->d_part_keys, 0, sizeof(unsigned long long) * (size_t)c->items_cap * c->key_stride) == cudaSuccess &&
+         talon::expand_setup(c) == TALON_OK && talon::attention_mma_setup() == TALON_OK &&
+         (c->k_cap > 32 || talon::expand_fused_setup(c) == TALON_OK);
   }
   if (!ok) {
     std::fprintf(stderr, "talon: context creation failed: %s\n", cudaGetErrorString(cudaGetLastError()));
@@ -149,7 +153,7 @@ talon_status talon_destroy(talon_ctx *c) {
   if (!c) return TALON_OK;
   cudaSetDevice(c->device);
   cudaFree(c->d_status); cudaFree(c->d_prefix_len); cudaFree(c->d_part_keys); cudaFree(c->d_part_ms);
-  cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_argmax);
+  cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_seq_count); cudaFree(c->d_argmax);
   cudaFree(c->d_target_tok); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
   talon_timing_enable(c, 0, 0u);

@@ -584,11 +584,12 @@ select_layer_kernel(SelectArgs a) {
 // ---------------------------------------------------------------------------------------
 __global__ void reset_kernel(talon_tree t, const int32_t *root_tok, const int32_t *prefix_len,
                              int32_t *prefix_copy, int B, int N, int W, int lo_stride, int *status,
-                             unsigned int *row_count, int rows_cap) {
+                             unsigned int *row_count, int rows_cap, unsigned int *seq_count) {
   const int gid = blockIdx.x * blockDim.x + threadIdx.x;
   const int stride = gridDim.x * blockDim.x;
   if (gid == 0) *status = 0;
   for (int i = gid; i < rows_cap; i += stride) row_count[i] = 0u;
+  for (int i = gid; i < B; i += stride) seq_count[i] = 0u;
   for (int b = gid; b < B; b += stride) {
     const size_t nb = (size_t)b * N;
     t.n_nodes[b] = 1;
@@ -671,7 +672,7 @@ talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root
   if (blocks < 1) blocks = 1;
   LaunchTimer lt(c, TALON_K_RESET, st);
   reset_kernel<<<blocks, threads, 0, st>>>(*t, root_tok, prefix_len, c->d_prefix_len, B, c->p.budget, c->W,
-                                           c->p.max_depth + 2, c->d_status, c->d_row_count, c->rows_cap);
+                                           c->p.max_depth + 2, c->d_status, c->d_row_count, c->rows_cap, c->d_seq_count);
   c->launches += 1;
   return cudaGetLastError() == cudaSuccess ? TALON_OK : TALON_ERR_CUDA;
 }
@@ -680,6 +681,8 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
                            int rows_per_seq, int layout, cudaStream_t st) {
   const int d = c->layers_run;
   const int fub = frontier_upper_bound(c, d);
+  if (c->k_cap <= 32)
+    return launch_expand_fused(c, t, logits, row_stride, rows_per_seq, layout, c->B * fub, st);
   long long max_items = (long long)c->B * fub * EXP_MAX_SPLITS;
   int grid = c->exp_grid;
   if (max_items < grid) grid = (int)max_items;

@@ -1,0 +1,727 @@
+// Adaptive draft-tree expansion (Algorithm 2 of the paper; Eq. 2-5) as ONE kernel per layer,
+// for per-parent candidate caps k <= 32 (the usual case: the paper's K is 10).
+//
+// Streaming phase.  The frontier's fp32 logit rows are cut into chunks, one CTA per chunk at a
+// time.  In a single read of its chunk a CTA produces the chunk's share of the softmax
+// normaliser of Eq. 3 (running maximum and sum of exponentials) and the chunk's k largest
+// logits with their token ids.  Each warp keeps a sorted list of its best k keys across its 32
+// lanes plus a small queue of elements that passed the current threshold; a full queue is
+// folded into the list with a bitonic sort and merge, which also raises the threshold.
+//
+// Selection phase.  The CTA that finishes the last chunk of a sequence merges that sequence's
+// chunk results into per-row top-k lists and log-sum-exps, scores the pooled candidates with
+// log p(u) = log p(v) + log P(w | v) (Eq. 2-3), applies Top-K (Eq. 5) or the confidence gate
+// p(u) >= mu * max p (Eq. 4), truncates to the remaining budget, and appends the survivors with
+// parent links, depths, scores and ancestor-mask rows.  Nothing returns to the host in between.
+#include <math_constants.h>
+
+#include "talon_internal.cuh"
+
+namespace talon {
+
+namespace {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr float LOG2E_F = 1.4426950408889634f;
+typedef unsigned long long u64;
+
+struct FusedArgs {
+  const float *logits;
+  int64_t row_stride;
+  int rows_per_seq, layout;
+  talon_tree t;
+  int lo_stride;
+  int B, N, W, V, d, k, key_stride, target_items, max_splits;
+  int root_topk, init_layers;
+  double log_mu;
+  u64 *part_keys;          // [items, key_stride]  per-chunk top-k, descending
+  float2 *part_ms;         // [items]              per-chunk (max, sum of exp)
+  unsigned int *seq_count; // [B]                  chunks finished per sequence (zero between layers)
+  int *status;
+};
+
+__device__ inline u64 shfl_u64(u64 v, int src) { return __shfl_sync(FULL, v, src); }
+__device__ inline u64 shfl_xor_u64(u64 v, int m) { return __shfl_xor_sync(FULL, v, m); }
+__device__ inline u64 umax64(u64 a, u64 b) { return a > b ? a : b; }
+__device__ inline u64 umin64(u64 a, u64 b) { return a < b ? a : b; }
+
+__device__ inline u64 warp_max_u64(u64 v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v = umax64(v, shfl_xor_u64(v, o));
+  return v;
+}
+
+// bitonic sort of one key per lane, descending by lane index
+__device__ inline u64 warp_sort_desc(u64 x, int lane) {
+#pragma unroll
+  for (int sz = 2; sz <= 32; sz <<= 1) {
+#pragma unroll
+    for (int j = sz >> 1; j > 0; j >>= 1) {
+      const u64 o = shfl_xor_u64(x, j);
+      const bool keep_max = (((lane & j) == 0) == ((lane & sz) == 0));
+      x = keep_max ? umax64(x, o) : umin64(x, o);
+    }
+  }
+  return x;
+}
+
+// list (descending across lanes) <- the 32 largest of list U q, q unsorted
+__device__ inline u64 warp_merge_desc(u64 list, u64 q, int lane) {
+  q = warp_sort_desc(q, lane);
+  u64 x = umax64(list, shfl_u64(q, 31 - lane));     // bitonic sequence holding the 32 largest
+#pragma unroll
+  for (int j = 16; j > 0; j >>= 1) {
+    const u64 o = shfl_xor_u64(x, j);
+    x = ((lane & j) == 0) ? umax64(x, o) : umin64(x, o);
+  }
+  return x;
+}
+
+// Folds the first 32 queued keys into the warp's list, moves the rest of the queue to its front
+// and raises the threshold to the list's k-th key.
+__device__ __forceinline__ void fold_queue(u64 &list, int &qn, float &thr_f, u64 *queue, float thr0, int k,
+                                           int lane) {
+  list = warp_merge_desc(list, queue[lane], lane);
+  const u64 rest = queue[32 + lane];
+  __syncwarp();
+  qn -= 32;
+  if (lane < qn) queue[lane] = rest;
+  __syncwarp();
+  const u64 kth = shfl_u64(list, k - 1);
+  if (kth) thr_f = fmaxf(thr0, key_logit(kth));
+}
+
+// Exclusive scan of the per-sequence frontier sizes: s_base[b] = first packed row of sequence
+// b, s_base[B] = total rows.  A sequence whose tree is full has no rows.
+__device__ void frontier_bases(const FusedArgs &a, int *s_base, int *s_warp) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (a.B <= 32) {
+    if (warp == 0) {
+      int f = 0;
+      if (lane < a.B && a.t.n_nodes[lane] < a.N) {
+        f = a.t.layer_off[lane * a.lo_stride + a.d + 1] - a.t.layer_off[lane * a.lo_stride + a.d];
+        f = max(f, 0);
+      }
+      int inc = f;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += t;
+      }
+      if (lane < a.B) s_base[lane] = inc - f;
+      if (lane == a.B - 1) s_base[a.B] = inc;
+    }
+    __syncthreads();
+    return;
+  }
+  constexpr int PER = (MAX_BATCH + EXP_THREADS - 1) / EXP_THREADS;
+  int f[PER];
+  int sum = 0;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int b = tid * PER + i;
+    int v = 0;
+    if (b < a.B && a.t.n_nodes[b] < a.N) {
+      v = a.t.layer_off[b * a.lo_stride + a.d + 1] - a.t.layer_off[b * a.lo_stride + a.d];
+      v = max(v, 0);
+    }
+    f[i] = v;
+    sum += v;
+  }
+  int inc = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(FULL, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    const int w = lane < EXP_WARPS ? s_warp[lane] : 0;
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(FULL, winc, o);
+      if (lane >= o) winc += t;
+    }
+    if (lane < EXP_WARPS) s_warp[lane] = winc - w;
+    if (lane == EXP_WARPS - 1) s_base[a.B] = winc;
+  }
+  __syncthreads();
+  int run = s_warp[warp] + inc - sum;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int b = tid * PER + i;
+    if (b < a.B) s_base[b] = run;
+    run += f[i];
+  }
+  __syncthreads();
+}
+
+__device__ inline int seq_of_row(const int *s_base, int B, int row) {
+  int lo = 0, hi = B;   // s_base[lo] <= row < s_base[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (s_base[mid] <= row) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ inline u64 f64_ord(double x) {
+  const u64 b = (u64)__double_as_longlong(x);
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+__device__ inline double f64_unord(u64 o) {
+  const u64 b = (o >> 63) ? (o & 0x7FFFFFFFFFFFFFFFull) : ~o;
+  return __longlong_as_double((long long)b);
+}
+
+// Where a packed frontier row lives: sequence, index inside that sequence's frontier, tree
+// node, frontier size and first packed row of the sequence.
+struct RowLoc { int b, j, node, F, row0; };
+
+// Frontier geometry of the layer.  For B <= 32 every warp holds it in registers (lane b = sequence
+// b) and needs no shared memory or barrier; larger batches use a block-wide scan.
+struct Frontier {
+  int base_l, f_l, lo_l;     // B <= 32: this lane's sequence
+  int total;
+  bool in_regs;
+  const int *s_base;
+};
+
+__device__ inline RowLoc locate_row(const FusedArgs &a, const Frontier &fr, int row) {
+  RowLoc r;
+  const int lane = threadIdx.x & 31;
+  if (fr.in_regs) {
+    // the last sequence whose first row is <= row (bases never decrease, empty sequences share
+    // their base with the next one)
+    const unsigned m = __ballot_sync(FULL, lane < a.B && fr.base_l <= row);
+    r.b = 31 - __clz(m);
+    r.row0 = __shfl_sync(FULL, fr.base_l, r.b);
+    r.F = __shfl_sync(FULL, fr.f_l, r.b);
+    r.j = row - r.row0;
+    r.node = __shfl_sync(FULL, fr.lo_l, r.b) + r.j;
+  } else {
+    r.b = seq_of_row(fr.s_base, a.B, row);
+    r.row0 = fr.s_base[r.b];
+    r.F = fr.s_base[r.b + 1] - r.row0;
+    r.j = row - r.row0;
+    r.node = a.t.layer_off[r.b * a.lo_stride + a.d] + r.j;
+  }
+  return r;
+}
+
+// Shared-memory carve-up of the selection phase.
+struct TailSmem {
+  u64 *stage;        // [EXP_WARPS][FX_STAGE]  chunk lists of the row a warp is merging
+  u64 *row_keys;     // [N-1][k]               per-row top-k keys, descending
+  double *score;     // [N-1][k]               log p(u) of each pooled candidate
+  double *row_t;     // [N-1]                  sum of exponentials, then the row's log-sum-exp
+  double *row_ps;    // [N-1]                  log p(v) of the row's parent
+  u64 *row_mask;     // [N-1][W]               ancestor mask of the row's parent
+  float *row_m;      // [N-1]
+  int *row_cnt, *row_off;   // [N-1]
+  unsigned char *state;     // [N-1][k]        bit0 eligible, bit2 selected
+};
+
+__device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int row0, int F, int S,
+                            u64 *s_anchor, int *s_cnt, int *s_bad) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k = a.k, ks = a.key_stride;
+  const int n = a.t.n_nodes[b];
+  const int lo = a.t.layer_off[b * a.lo_stride + a.d];
+  const int R = a.N - n;
+  const int ke = min(k, R);                 // a parent can place at most R children
+  const size_t nb = (size_t)b * a.N;
+  if (tid == 0) { *s_anchor = 0ull; *s_cnt = 0; *s_bad = 0; }
+
+  // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys ----
+  for (int j = warp; j < F; j += EXP_WARPS) {
+    const size_t item0 = (size_t)(row0 + j) * S;
+    // everything this row needs from global memory, issued together
+    float2 ms[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int c = lane + 32 * i;
+      ms[i] = (c < S) ? __ldcg(a.part_ms + item0 + c) : make_float2(-CUDART_INF_F, 0.f);
+    }
+    u64 *st = sm.stage + warp * FX_STAGE;
+    u64 *rk = sm.row_keys + (size_t)j * k;
+    const int nk = S * ks;                  // padding slots (p >= k) always hold zero
+    if (S == 1) {
+      if (lane < k) rk[lane] = __ldcg(a.part_keys + item0 * ks + lane);
+    } else {
+      for (int idx = lane; idx < nk; idx += 32) st[idx] = __ldcg(a.part_keys + item0 * ks + idx);
+    }
+    if (lane == 0) sm.row_ps[j] = a.t.score[nb + lo + j];
+    if (lane < a.W) sm.row_mask[j * a.W + lane] = a.t.mask[(nb + lo + j) * a.W + lane];
+
+    float mx = fmaxf(ms[0].x, ms[1].x);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+    double t = 0.0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      if (ms[i].y != ms[i].y) t += (double)ms[i].y;                       // NaN or +inf logit in the chunk
+      else if (ms[i].x > -CUDART_INF_F) t += (double)ms[i].y * (double)exp2f((ms[i].x - mx) * LOG2E_F);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
+    if (lane == 0) { sm.row_m[j] = mx; sm.row_t[j] = t; }
+    if (S == 1) continue;
+
+    if (lane < k) rk[lane] = 0ull;
+    __syncwarp();
+    // Two lower bounds of the row's k-th best key: the best k-th key of any one chunk, and the
+    // k-th best of the chunk heads (k different chunks each hold a key at least that large).
+    u64 tau = 0ull;
+    for (int c = lane; c < S; c += 32) {
+      tau = umax64(tau, st[c * ks + k - 1]);
+      if (S >= k) {
+        const u64 h = st[c * ks];
+        int cnt = 0;
+        for (int o = 0; o < S; ++o) cnt += (st[o * ks] > h) ? 1 : 0;
+        if (cnt == k - 1) tau = umax64(tau, h);
+      }
+    }
+    tau = warp_max_u64(tau);
+    // compact the keys that reach the bound to the front of the staging area
+    int mine = 0;
+    for (int idx = lane; idx < nk; idx += 32) {
+      const u64 key = st[idx];
+      mine += (key != 0ull && key >= tau) ? 1 : 0;
+    }
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(FULL, inc, o);
+      if (lane >= o) inc += v;
+    }
+    const int ns = __shfl_sync(FULL, inc, 31);
+    u64 *sv = st + nk;                       // survivors go behind the lists (nk <= FX_STAGE / 2)
+    int pos = inc - mine;
+    for (int idx = lane; idx < nk; idx += 32) {
+      const u64 key = st[idx];
+      if (key != 0ull && key >= tau) sv[pos++] = key;
+    }
+    __syncwarp();
+    // rank by counting (keys are unique)
+    for (int i = lane; i < ns; i += 32) {
+      const u64 key = sv[i];
+      int r = 0;
+      for (int o = 0; o < ns; ++o) r += (sv[o] > key) ? 1 : 0;
+      if (r < k) rk[r] = key;
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+
+  // ---- log-sum-exp of every row ----
+  for (int j = tid; j < F; j += EXP_THREADS) {
+    const double t = sm.row_t[j];
+    const float m = sm.row_m[j];
+    double lse = (double)m + log(t);
+    if (!(t > 0.0) || !(m < CUDART_INF_F) || lse != lse) {
+      lse = CUDART_NAN;
+      *s_bad = 1;
+      atomicOr(a.status, STATUS_NONFINITE);
+    }
+    sm.row_t[j] = lse;
+    sm.row_cnt[j] = 0;
+  }
+  __syncthreads();
+  if (*s_bad) {            // a frontier row was not finite: this sequence adds nothing
+    if (tid == 0) a.t.layer_off[b * a.lo_stride + a.d + 2] = n;
+    return;
+  }
+
+  // ---- pool: log p(u) = log p(v) + (z_w - lse_v)   (Eq. 2-3) ----
+  const int C = F * k;
+  for (int c = tid; c < C; c += EXP_THREADS) {
+    const int j = c / k, i = c - j * k;
+    const u64 key = sm.row_keys[c];
+    double s = -CUDART_INF;
+    if (i < ke && key != 0ull) s = sm.row_ps[j] + ((double)key_logit(key) - sm.row_t[j]);
+    const bool ok = (s > -CUDART_INF) && (s == s);
+    if (!ok) s = -CUDART_INF;
+    sm.score[c] = s;
+    sm.state[c] = ok ? 1 : 0;
+    if (ok && i == 0) atomicMax(s_anchor, f64_ord(s));        // rows are sorted: heads carry the maxima
+  }
+  __syncthreads();
+
+  // ---- eligibility: Top-K layers take every candidate, gated layers Eq. 4 ----
+  const bool init = a.d < a.init_layers;
+  double thr = -CUDART_INF;
+  if (!init && *s_anchor != 0ull) thr = a.log_mu + f64_unord(*s_anchor);
+  int local = 0;
+  for (int c = tid; c < C; c += EXP_THREADS) {
+    unsigned char stt = sm.state[c];
+    if (stt && !init && !(sm.score[c] >= thr)) stt = 0;
+    sm.state[c] = stt;
+    local += stt;
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(FULL, local, o);
+  if (lane == 0 && local) atomicAdd(s_cnt, local);
+  __syncthreads();
+  const int eligible = *s_cnt;
+  const int want = init ? min(a.root_topk, R) : R;
+  const int n_sel = min(eligible, want);
+
+  // ---- budget truncation: rank among all candidates by (score desc, parent asc, token asc).
+  // Every row is sorted that way already, so a rank is a sum of binary searches. ----
+  for (int c = tid; c < C; c += EXP_THREADS) {
+    if (!sm.state[c]) continue;
+    bool sel = true;
+    if (eligible > want) {
+      const int j = c / k, i = c - j * k;
+      const double s = sm.score[c];
+      int rank = i;
+      for (int o = 0; o < F; ++o) {
+        if (o == j) continue;
+        const double *sc = sm.score + o * k;
+        const bool before = o < j;
+        int l = 0, h = ke;
+        while (l < h) {
+          const int mid = (l + h) >> 1;
+          const double v = sc[mid];
+          if (v > s || (v == s && before)) l = mid + 1; else h = mid;
+        }
+        rank += l;
+      }
+      sel = rank < want;
+    }
+    if (sel) {
+      sm.state[c] = 5;
+      atomicAdd(&sm.row_cnt[c / k], 1);
+    }
+  }
+  __syncthreads();
+
+  // ---- append in storage order: (parent asc, token asc) ----
+  if (warp == 0) {
+    int v[4], sum = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const int jj = lane * 4 + i; v[i] = jj < F ? sm.row_cnt[jj] : 0; sum += v[i]; }
+    int inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(FULL, inc, o);
+      if (lane >= o) inc += t;
+    }
+    int run = inc - sum;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const int jj = lane * 4 + i; if (jj < F) sm.row_off[jj] = run; run += v[i]; }
+  }
+  __syncthreads();
+  for (int c = tid; c < C; c += EXP_THREADS) {
+    if (!(sm.state[c] & 4)) continue;
+    const int j = c / k;
+    const int tok = (int)key_tok(sm.row_keys[c]);
+    int r = 0;
+    for (int i = 0; i < ke; ++i) {
+      const int o = j * k + i;
+      r += ((sm.state[o] & 4) && (int)key_tok(sm.row_keys[o]) < tok) ? 1 : 0;
+    }
+    const int node = n + sm.row_off[j] + r;
+    a.t.token[nb + node] = tok;
+    a.t.parent[nb + node] = lo + j;
+    a.t.depth[nb + node] = a.d + 1;
+    a.t.score[nb + node] = sm.score[c];
+    for (int w = 0; w < a.W; ++w) {
+      u64 m = sm.row_mask[j * a.W + w];
+      if ((node >> 6) == w) m |= 1ull << (node & 63);
+      a.t.mask[(nb + node) * a.W + w] = m;
+    }
+  }
+  if (tid == 0) {
+    a.t.n_nodes[b] = n + n_sel;
+    a.t.layer_off[b * a.lo_stride + a.d + 2] = n + n_sel;
+  }
+}
+
+__global__ void __launch_bounds__(EXP_THREADS)
+expand_fused_kernel(FusedArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ u64 s_queue[EXP_WARPS][FX_QCAP];       // per-warp queues of keys above the threshold
+  __shared__ u64 s_pool[EXP_WARPS * 32];            // the chunk's candidates: at most 32 per warp
+  __shared__ int s_base[MAX_BATCH + 1];
+  __shared__ int s_warp[EXP_WARPS];
+  __shared__ float s_m[EXP_WARPS], s_s[EXP_WARPS];
+  __shared__ u64 s_anchor;
+  __shared__ int s_pool_n, s_last, s_cnt, s_bad;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k = a.k;
+
+  // ---- frontier geometry ----
+  Frontier fr;
+  fr.in_regs = a.B <= 32;
+  fr.s_base = s_base;
+  fr.base_l = fr.f_l = fr.lo_l = 0;
+  if (fr.in_regs) {
+    if (lane < a.B) {
+      const int nn = a.t.n_nodes[lane];
+      fr.lo_l = a.t.layer_off[lane * a.lo_stride + a.d];
+      const int hi = a.t.layer_off[lane * a.lo_stride + a.d + 1];
+      fr.f_l = nn < a.N ? max(hi - fr.lo_l, 0) : 0;
+      if (fr.f_l == 0 && blockIdx.x == 0 && warp == 0)        // nothing to expand: close the layer
+        a.t.layer_off[lane * a.lo_stride + a.d + 2] = nn;
+    }
+    int inc = fr.f_l;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(FULL, inc, o);
+      if (lane >= o) inc += t;
+    }
+    fr.base_l = inc - fr.f_l;
+    fr.total = __shfl_sync(FULL, inc, 31);
+  } else {
+    frontier_bases(a, s_base, s_warp);
+    fr.total = s_base[a.B];
+    if (blockIdx.x == 0)
+      for (int b = tid; b < a.B; b += EXP_THREADS)
+        if (s_base[b + 1] == s_base[b]) a.t.layer_off[b * a.lo_stride + a.d + 2] = a.t.n_nodes[b];
+  }
+  if (tid == 0) s_pool_n = 0;
+  const LayerGeom g = make_geom(fr.total, a.V, a.target_items, a.max_splits, EXP_TILE);
+  const int n_items = fr.total * g.splits;
+  __syncthreads();
+
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int row = item / g.splits, chunk = item - row * g.splits;
+    const RowLoc rl = locate_row(a, fr, row);
+    int rsel = (a.layout == TALON_ROWS_BY_NODE) ? rl.node : rl.j;
+    if (rsel >= a.rows_per_seq) {               // caller reserved too few rows: stay in bounds, report
+      rsel = a.rows_per_seq - 1;
+      if (tid == 0) atomicOr(a.status, STATUS_CAPACITY);
+    }
+    const float *rowp = a.logits + ((int64_t)rl.b * a.rows_per_seq + rsel) * a.row_stride;
+    const int start = chunk * g.chunk_len;
+    const int end = min(a.V, start + g.chunk_len);
+
+    float m_t = -CUDART_INF_F, s_t = 0.f;
+    u64 list = 0ull;                 // lane p holds the warp's p-th best key so far (once folded)
+    bool folded = false;
+    int qn = 0;                      // keys waiting in this warp's queue (< 32 between tiles)
+    float thr0 = -CUDART_INF_F, thr_f = -CUDART_INF_F;
+    bool first = true;
+    u64 *queue = s_queue[warp];
+
+
+    for (int base = start; base < end; base += EXP_TILE) {
+      float v[EXP_UNROLL][EXP_VEC];
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u) {
+        const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+        if (idx + EXP_VEC <= end) {
+          const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
+          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+        } else {
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
+        }
+      }
+      float bm = -CUDART_INF_F;
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+        for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
+
+      if (first) {
+        first = false;
+        // k lane maxima are k distinct elements, so the k-th largest lane maximum is a lower
+        // bound of this warp's k-th largest element: nothing below it needs to be looked at.
+        int rank = 0;
+#pragma unroll
+        for (int l = 0; l < 32; ++l) {
+          const float o = __shfl_sync(FULL, bm, l);
+          rank += (o > bm) || (o == bm && l < lane);
+        }
+        const unsigned pick = __ballot_sync(FULL, rank == k - 1);
+        if (pick) thr0 = __shfl_sync(FULL, bm, __ffs(pick) - 1);
+        thr_f = thr0;
+      }
+      // running softmax normaliser of this thread's elements
+      if (bm > m_t) {
+        s_t *= exp2f((m_t - bm) * LOG2E_F);
+        m_t = bm;
+      }
+      if (m_t > -CUDART_INF_F) {
+        float acc = 0.f;
+#pragma unroll
+        for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - m_t) * LOG2E_F);
+        s_t += acc;
+      }
+      // top-k: elements that reach the threshold go to the warp's queue
+      int mine = 0;
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+        for (int e = 0; e < EXP_VEC; ++e)
+          mine += (v[u][e] >= thr_f && base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
+      if (!__any_sync(FULL, mine > 0)) continue;
+      int inc = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const int total = __shfl_sync(FULL, inc, 31);
+      if (total <= 32) {
+        int pos = qn + inc - mine;
+#pragma unroll
+        for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) {
+            const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+            if (v[u][e] >= thr_f && tok < end) queue[pos++] = cand_key(v[u][e], (uint32_t)tok);
+          }
+        qn += total;
+        __syncwarp();
+        if (qn >= 32) { fold_queue(list, qn, thr_f, queue, thr0, k, lane); folded = true; }
+      } else {
+        // many elements at or above the threshold (equal logits, or a cold threshold): one
+        // register slot at a time, folding whenever 32 keys are waiting
+#pragma unroll
+        for (int u = 0; u < EXP_UNROLL; ++u) {
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) {
+            const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+            const bool ok = v[u][e] >= thr_f && tok < end;
+            const unsigned mk = __ballot_sync(FULL, ok);
+            if (mk == 0u) continue;
+            if (ok) queue[qn + __popc(mk & ((1u << lane) - 1u))] = cand_key(v[u][e], (uint32_t)tok);
+            qn += __popc(mk);
+            __syncwarp();
+            if (qn >= 32) { fold_queue(list, qn, thr_f, queue, thr0, k, lane); folded = true; }
+          }
+        }
+      }
+    }
+
+    // ---- this warp's candidates -> the CTA pool; (max, sum) -> shared ----
+    int cnt_w = qn;
+    if (folded) {
+      if (qn > 0) list = warp_merge_desc(list, lane < qn ? queue[lane] : 0ull, lane);
+      cnt_w = __popc(__ballot_sync(FULL, lane < k && list != 0ull));
+    }
+    int pos = 0;
+    if (lane == 0) pos = atomicAdd(&s_pool_n, cnt_w);
+    pos = __shfl_sync(FULL, pos, 0);
+    if (lane < cnt_w) s_pool[pos + lane] = folded ? list : queue[lane];
+    float wm = m_t;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(FULL, wm, o));
+    // thread partial rescaled to the warp maximum; a NaN partial (NaN or +inf logit) propagates
+    float ws = (m_t > -CUDART_INF_F || s_t != s_t) ? s_t * exp2f((m_t - wm) * LOG2E_F) : 0.f;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
+    if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
+    __syncthreads();
+
+    // ---- the chunk's k best keys (rank by counting: keys are unique) and its (max, sum) ----
+    const int nc = s_pool_n;
+    if (tid < nc) {
+      const u64 key = s_pool[tid];
+      int r = 0;
+#pragma unroll 4
+      for (int o = 0; o < nc; ++o) r += (s_pool[o] > key) ? 1 : 0;
+      if (r < k) a.part_keys[(size_t)item * a.key_stride + r] = key;
+    }
+    if (tid >= nc && tid < k) a.part_keys[(size_t)item * a.key_stride + tid] = 0ull;
+    if (warp == EXP_WARPS - 1) {
+      const float mw = lane < EXP_WARPS ? s_m[lane] : -CUDART_INF_F;
+      const float sw = lane < EXP_WARPS ? s_s[lane] : 0.f;
+      float bmx = mw;
+#pragma unroll
+      for (int o = 4; o; o >>= 1) bmx = fmaxf(bmx, __shfl_xor_sync(FULL, bmx, o));
+      float tot = (mw > -CUDART_INF_F || sw != sw) ? sw * exp2f((mw - bmx) * LOG2E_F) : 0.f;
+#pragma unroll
+      for (int o = 4; o; o >>= 1) tot += __shfl_xor_sync(FULL, tot, o);
+      if (lane == 0) a.part_ms[item] = make_float2(bmx, tot);
+    }
+
+    // ---- the last chunk of a sequence runs that sequence's selection ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      s_pool_n = 0;
+      const unsigned prev = atomicAdd(&a.seq_count[rl.b], 1u);
+      s_last = (prev == (unsigned)(rl.F * g.splits) - 1u);
+      if (s_last) a.seq_count[rl.b] = 0u;            // ready for the next layer
+    }
+    __syncthreads();
+    if (!s_last) continue;
+    __threadfence();
+    TailSmem sm;
+    const int rows_max = a.N - 1;
+    unsigned char *p = smem_raw;
+    sm.stage = reinterpret_cast<u64 *>(p);            p += sizeof(u64) * EXP_WARPS * FX_STAGE;
+    sm.row_keys = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * k;
+    sm.score = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max * k;
+    sm.row_t = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max;
+    sm.row_ps = reinterpret_cast<double *>(p);        p += sizeof(double) * rows_max;
+    sm.row_mask = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * a.W;
+    sm.row_m = reinterpret_cast<float *>(p);          p += sizeof(float) * rows_max;
+    sm.row_cnt = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
+    sm.row_off = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
+    sm.state = p;
+    select_tail(a, sm, rl.b, rl.row0, rl.F, g.splits, &s_anchor, &s_cnt, &s_bad);
+  }
+}
+
+size_t fused_smem_bytes(const talon_ctx *c) {
+  const size_t rows = c->p.budget - 1, k = c->k_cap, W = c->W;
+  return sizeof(u64) * EXP_WARPS * FX_STAGE + rows * k * (8 + 8 + 1) + rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
+}
+
+}  // namespace
+
+int fused_max_splits(int key_stride) {
+  int s = FX_STAGE / (2 * key_stride);          // half of a warp's staging area stays free for survivors
+  return s > FX_MAX_SPLITS ? FX_MAX_SPLITS : (s < 1 ? 1 : s);
+}
+
+talon_status expand_fused_setup(talon_ctx *c) {
+  const size_t bytes = fused_smem_bytes(c);
+  if (cudaFuncSetAttribute(expand_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) !=
+      cudaSuccess)
+    return TALON_ERR_CUDA;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, expand_fused_kernel, EXP_THREADS, bytes) !=
+      cudaSuccess || per_sm < 1)
+    return TALON_ERR_CUDA;
+  if (per_sm > EXP_CTAS_PER_SM) per_sm = EXP_CTAS_PER_SM;
+  c->fused_grid = c->sm_count * per_sm;
+  return TALON_OK;
+}
+
+talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,
+                                 int rows_per_seq, int layout, int rows_bound, cudaStream_t st) {
+  FusedArgs a;
+  a.logits = logits; a.row_stride = row_stride; a.rows_per_seq = rows_per_seq; a.layout = layout;
+  a.t = *t; a.lo_stride = c->p.max_depth + 2;
+  a.B = c->B; a.N = c->p.budget; a.W = c->W; a.V = c->p.vocab; a.d = c->layers_run; a.k = c->k_cap;
+  a.key_stride = c->key_stride;
+  a.max_splits = fused_max_splits(c->key_stride);
+  long long max_items = (long long)rows_bound * a.max_splits;
+  int grid = c->fused_grid;
+  if (max_items < grid) grid = (int)max_items;
+  if (grid < 1) grid = 1;
+  a.target_items = c->fused_grid;
+  a.root_topk = c->p.root_topk; a.init_layers = c->p.init_layers; a.log_mu = c->log_mu;
+  a.part_keys = c->d_part_keys; a.part_ms = c->d_part_ms; a.seq_count = c->d_seq_count; a.status = c->d_status;
+  {
+    LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
+    expand_fused_kernel<<<grid, EXP_THREADS, fused_smem_bytes(c), st>>>(a);
+  }
+  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+  c->launches += 1;
+  return TALON_OK;
+}
+
+}  // namespace talon

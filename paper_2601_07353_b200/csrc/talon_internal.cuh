@@ -25,6 +25,10 @@ constexpr int EXP_CTAS_PER_SM = 4;
 constexpr int MAX_BUDGET = 128;
 constexpr int MAX_BATCH = 1024;
 constexpr int SEL_THREADS = 512;
+// fused expansion kernel (k <= 32)
+constexpr int FX_QCAP = 64;                // keys a warp's queue can hold
+constexpr int FX_STAGE = 512;              // keys a warp stages while merging one row's chunk lists
+constexpr int FX_MAX_SPLITS = 64;          // chunks per row, at most
 
 // Order-preserving map fp32 -> u32 (larger float <=> larger integer; -inf > 0).
 __host__ __device__ inline uint32_t f32_ord(float f) {
@@ -58,14 +62,16 @@ struct LayerGeom {
   int chunk_len;    // elements per chunk (multiple of EXP_CHUNK_ALIGN)
 };
 
-__host__ __device__ inline LayerGeom make_geom(int total_rows, int vocab, int target_items) {
+__host__ __device__ inline LayerGeom make_geom(int total_rows, int vocab, int target_items,
+                                               int max_splits = EXP_MAX_SPLITS, int min_chunk = EXP_CHUNK_ALIGN) {
   LayerGeom g;
   g.total_rows = total_rows;
   int want = total_rows > 0 ? (target_items + total_rows - 1) / total_rows : 1;
   if (want < 1) want = 1;
-  if (want > EXP_MAX_SPLITS) want = EXP_MAX_SPLITS;
+  if (want > max_splits) want = max_splits;
   int len = (vocab + want - 1) / want;
   len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
+  if (len < min_chunk) len = min_chunk;
   g.chunk_len = len;
   g.splits = (vocab + len - 1) / len;
   return g;
@@ -98,6 +104,8 @@ struct talon_ctx {
   unsigned long long *d_row_keys;    // [rows_cap, key_stride]   per-row top-k
   double *d_row_lse;                 // [rows_cap]               per-row log-sum-exp
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
+  unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
+  int fused_grid;                    // CTAs of the fused kernel at full width
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
   int32_t *d_target_tok;             // [batch_max * N]
@@ -147,5 +155,8 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                            int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st);
 size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems);
+talon_status expand_fused_setup(talon_ctx *c);
+talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,
+                                 int rows_per_seq, int layout, int rows_bound, cudaStream_t st);
 
 }  // namespace talon
