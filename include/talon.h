@@ -139,13 +139,16 @@ talon_status talon_build_tree(talon_ctx *ctx, const talon_tree *tree, uint8_t *d
  *           strides multiples of 8)
  *  k_tree, v_tree      [B, N, Hkv, Dh] contiguous: keys/values of the tree tokens themselves
  *  kv_start device [B] int64 token offsets of each sequence's block (ragged or padded)
+ *  kv_tokens           tokens allocated in k_prefix / v_prefix (host value): reads stop there, so
+ *                      kv_start[b] + L_b <= kv_tokens must hold; memory between L_b and the next
+ *                      multiple of 128 tokens may be read but never influences the result
  *  max_prefix_len      host upper bound of the prefix lengths given to talon_reset
  *  out      [B, N, Hq, Dh] contiguous; rows of unused node slots are written as zeros
  * Rotary embedding is the caller's business: Q/K arrive already rotated. */
 talon_status talon_tree_attention(talon_ctx *ctx, const talon_tree *tree, const void *q,
                                   const void *k_prefix, const void *v_prefix,
                                   const void *k_tree, const void *v_tree,
-                                  const int64_t *kv_start, int64_t kv_stride_t,
+                                  const int64_t *kv_start, int64_t kv_tokens, int64_t kv_stride_t,
                                   int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale,
                                   void *out, void *stream);
 
@@ -201,8 +204,9 @@ talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const
                         const int32_t *prefix_len, const float *draft_logits,
                         int64_t draft_row_stride, int32_t n_layers, const void *q,
                         const void *k_prefix, const void *v_prefix, const void *k_tree,
-                        const void *v_tree, const int64_t *kv_start, int64_t kv_stride_t,
-                        int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
+                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len,
+                        float sm_scale, void *out,
                         const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
                         int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
                         void *stream);

@@ -10,6 +10,7 @@
 namespace talon {
 talon_status expand_setup(talon_ctx *c);
 talon_status attention_mma_setup();
+talon_status attention_tc_setup();
 }  // namespace talon
 
 // Device staging for talon_step_host.
@@ -138,6 +139,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
          cudaMemset(c->d_seq_count, 0, sizeof(unsigned int) * (size_t)p->batch_max) == cudaSuccess &&
          cudaMemset(c->d_part_keys, 0, sizeof(unsigned long long) * (size_t)c->items_cap * c->key_stride) == cudaSuccess &&
          talon::expand_setup(c) == TALON_OK && talon::attention_mma_setup() == TALON_OK &&
+         talon::attention_tc_setup() == TALON_OK &&
          (c->k_cap > 32 || talon::expand_fused_setup(c) == TALON_OK);
   }
   if (!ok) {
@@ -194,10 +196,12 @@ talon_status talon_build_tree(talon_ctx *c, const talon_tree *t, uint8_t *dense_
 
 talon_status talon_tree_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *k_prefix,
                                   const void *v_prefix, const void *k_tree, const void *v_tree,
-                                  const int64_t *kv_start, int64_t kv_stride_t, int64_t kv_stride_h,
-                                  int32_t max_prefix_len, float sm_scale, void *out, void *stream) {
+                                  const int64_t *kv_start, int64_t kv_tokens, int64_t kv_stride_t,
+                                  int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                                  void *stream) {
   if (!c || !tree_complete(t) || !q || !k_tree || !v_tree || !kv_start || !out) return TALON_ERR_INVALID_ARG;
-  if (c->B < 1 || max_prefix_len < 0) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || max_prefix_len < 0 || kv_tokens < 0 || kv_tokens > 0x7FFFFFFFll) return TALON_ERR_INVALID_ARG;
+  if (max_prefix_len > kv_tokens) return TALON_ERR_INVALID_ARG;
   if (max_prefix_len > 0 && (!k_prefix || !v_prefix)) return TALON_ERR_INVALID_ARG;
   if ((kv_stride_t & 7) || (kv_stride_h & 7) || kv_stride_t < 0 || kv_stride_h < 0) return TALON_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_prefix) || !aligned16(v_prefix) || !aligned16(k_tree) || !aligned16(v_tree) ||
@@ -205,8 +209,8 @@ talon_status talon_tree_attention(talon_ctx *c, const talon_tree *t, const void 
     return TALON_ERR_INVALID_ARG;
   if (!(sm_scale == sm_scale)) return TALON_ERR_INVALID_ARG;
   return talon::launch_attention(c, t, q, k_prefix ? k_prefix : k_tree, v_prefix ? v_prefix : v_tree, k_tree,
-                                 v_tree, kv_start, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out,
-                                 (cudaStream_t)stream);
+                                 v_tree, kv_start, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale,
+                                 out, (cudaStream_t)stream);
 }
 
 talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
@@ -286,8 +290,8 @@ talon_status talon_timing_read(talon_ctx *c, void *stream, double *ms, int64_t *
 talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
                         const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
                         int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
-                        const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_stride_t,
-                        int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
+                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
                         const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
                         int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok, void *stream) {
   if (!c) return TALON_ERR_INVALID_ARG;
@@ -297,7 +301,7 @@ talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int3
     r = talon_expand_layer(c, t, draft_logits, draft_row_stride, c->p.budget, TALON_ROWS_BY_NODE, stream);
   if (r == TALON_OK) r = talon_build_tree(c, t, nullptr, stream);
   if (r == TALON_OK)
-    r = talon_tree_attention(c, t, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_stride_t, kv_stride_h,
+    r = talon_tree_attention(c, t, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_tokens, kv_stride_t, kv_stride_h,
                              max_prefix_len, sm_scale, out, stream);
   if (r == TALON_OK)
     r = talon_accept(c, t, target_logits, target_row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
@@ -393,7 +397,7 @@ talon_status talon_step_host(talon_ctx *c, int32_t B, const int32_t *root_tok, c
     r = talon_expand_layer(c, &s->tree, s->draft, (int64_t)V, (int32_t)N, TALON_ROWS_BY_NODE, stream);
   if (r == TALON_OK) r = talon_build_tree(c, &s->tree, nullptr, stream);
   if (r == TALON_OK)
-    r = talon_tree_attention(c, &s->tree, s->q, s->kp, s->vp, s->kt, s->vt, s->kv_start,
+    r = talon_tree_attention(c, &s->tree, s->q, s->kp, s->vp, s->kt, s->vt, s->kv_start, s->prefix_tokens,
                              (int64_t)p.n_kv_heads * Dh, (int64_t)Dh, max_len, sm_scale, s->out, stream);
   if (r == TALON_OK)
     r = talon_accept(c, &s->tree, s->target, (int64_t)V, nullptr, s->accept_len, s->accept_nodes, s->bonus, stream);

@@ -15,11 +15,11 @@
 namespace talon {
 
 constexpr int AT_THREADS = 256;
-constexpr int AT_WARPS = 8;
 constexpr int AT_BM = 128;     // packed query rows per CTA (16 per warp)
 constexpr int AT_BN = 64;      // keys per tile
 constexpr int AT_D = 128;      // head dimension
 constexpr int AT_TILE_BYTES = AT_BN * AT_D * 2;
+constexpr int TC_MIN_TILES_PER_CTA = 4;   // split-KV of the tensor-core path: key tiles a CTA should at least own
 constexpr int AT_SMEM = AT_BM * AT_D * 2 + 4 * AT_TILE_BYTES;   // Q + 2 stages of (K, V)
 
 struct AttnArgs {
@@ -342,8 +342,8 @@ talon_status attention_mma_setup() {
 }
 
 talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
-                              const void *kt, const void *vt, const int64_t *kv_start, int64_t stride_t,
-                              int64_t stride_h, int max_prefix_len, float sm_scale, void *out,
+                              const void *kt, const void *vt, const int64_t *kv_start, int64_t kv_tokens,
+                              int64_t stride_t, int64_t stride_h, int max_prefix_len, float sm_scale, void *out,
                               cudaStream_t st) {
   AttnArgs a;
   a.q = (const __nv_bfloat16 *)q; a.kp = (const __nv_bfloat16 *)kp; a.vp = (const __nv_bfloat16 *)vp;
@@ -355,6 +355,34 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   a.m_blocks = attn_m_blocks(c);
   a.out = (__nv_bfloat16 *)out; a.part_o = c->d_attn_o; a.part_ml = c->d_attn_ml;
+
+  if (attention_tc_supported(c, stride_t, stride_h, sm_scale)) {
+    // tensor-core path: CTAs own two 128-row query tiles and 128-key tiles
+    const int pairs = (a.m_blocks + 1) / 2;
+    const int ctas = pairs * c->B * a.Hkv;
+    const int tiles = (max_prefix_len + 127) / 128 + (a.N + 127) / 128;
+    int sp = 1;
+    if (ctas < c->sm_count) {
+      sp = c->sm_count / ctas;
+      const int by_tiles = (tiles + TC_MIN_TILES_PER_CTA - 1) / TC_MIN_TILES_PER_CTA;
+      if (sp > by_tiles) sp = by_tiles;
+      if (sp < 1) sp = 1;
+    }
+    while (sp > 1 && (size_t)a.m_blocks * c->B * a.Hkv * sp * AT_BM > c->attn_ml_elems) --sp;
+    a.splits = sp;
+    talon_status r = launch_attention_tc(c, t, q, kp, vp, kt, vt, kv_start, stride_t, stride_h, kv_tokens,
+                                         max_prefix_len, sm_scale, out, sp, a.m_blocks, st);
+    if (r != TALON_OK) return r;
+    if (sp > 1) {
+      const int64_t rows = (int64_t)c->B * a.Hkv * a.g * a.N;
+      const int wpb = 8;
+      LaunchTimer lt(c, TALON_K_COMBINE, st);
+      attention_combine_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(a);
+      if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+      c->launches += 1;
+    }
+    return TALON_OK;
+  }
 
   const int base = a.m_blocks * c->B * a.Hkv;
   const int max_tiles = (max_prefix_len + AT_BN - 1) / AT_BN + (a.N + AT_BN - 1) / AT_BN;

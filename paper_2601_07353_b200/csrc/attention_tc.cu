@@ -1,0 +1,598 @@
+// Tree attention (verification forward of Appendix B) on the 5th-generation tensor cores.
+//
+// Work split.  For sequence b and kv head h the g = Hq/Hkv query heads of all N tree nodes are
+// packed into one [g*N, 128] query matrix (row = node * g + head-in-group), so every K/V tile
+// is read once for the whole group.  A CTA owns up to two 128-row query tiles and a range of
+// 128-key tiles of the key axis (the L_b prefix keys, then the tree keys); with several
+// ranges per (b, h) a second kernel merges the partial results (split-KV).
+//
+// Roles inside a CTA (320 threads):
+//   warps 0-3, 4-7  softmax of query tile 0 / 1: thread r owns row r.  It reads its row of
+//                   S = Q K^T from tensor memory (tcgen05.ld), applies the ragged-length or
+//                   ancestor-bitmask visibility, keeps a running maximum and sum, and writes
+//                   P = exp2(S*scale - max) as bf16 back to tensor memory over S (tcgen05.st).
+//                   The running maximum is only raised when it grows by more than 2^8, so the
+//                   accumulator in tensor memory is rescaled rarely (the final division by the
+//                   running sum makes any reference maximum exact).
+//   warp 8          producer: TMA loads of Q (once) and of the K / V tiles into a ring of
+//                   128-byte-swizzled shared-memory stages (no multicast).
+//   warp 9          one thread issues tcgen05.mma: S_i = Q_i K^T (both operands in shared
+//                   memory) and O_i += P_i V (P from tensor memory, V from shared memory), with
+//                   tcgen05.commit arriving on mbarriers that the other roles wait on.
+// Every wait is bounded: a role that gives up raises a flag that makes the other roles leave
+// too, tensor memory is released, and the device status word reports a timeout.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include <cstdio>
+#include <cstring>
+
+#include "talon_internal.cuh"
+
+namespace talon {
+
+namespace {
+
+constexpr int TC_BN = 128;                 // keys per tile
+constexpr int TC_D = 128;                  // head dimension
+constexpr int TC_MT = 128;                 // query rows per tile
+constexpr int TC_STAGES = 2;               // K and V ring depth
+constexpr int TC_THREADS = 320;
+constexpr int TC_TILE_BYTES = TC_BN * TC_D * 2;      // 32 KB: one K, V or Q tile
+constexpr int TC_HALF_BYTES = TC_BN * 64 * 2;        // 16 KB: the 64-element half of a tile
+constexpr int TC_NBARS = 16;
+constexpr int TC_SMEM = (2 + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 + TC_NBARS * 8 + 64;
+constexpr uint32_t TC_TMEM_COLS = 512;     // O0 | O1 | S0 | S1, 128 fp32 columns each
+constexpr float TC_RESCALE_GAP = 8.f;      // raise the reference maximum only beyond 2^8
+constexpr long long TC_WAIT_CYCLES = 4000000000ll;   // ~2 s: far beyond any legitimate wait
+
+// barrier slots
+enum { B_Q = 0, B_KFULL = 1, B_VFULL = 3, B_KEMPTY = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_ODONE = 13 };
+
+struct TcArgs {
+  const int64_t *kv_start;
+  const int32_t *prefix_len, *n_nodes;
+  const unsigned long long *mask;
+  int B, N, W, Hq, Hkv, g;
+  float scale_log2;
+  int splits, m_blocks;
+  __nv_bfloat16 *out;
+  float *part_o;
+  float2 *part_ml;
+  int *status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ inline void mbar_arrive(uint32_t bar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
+}
+__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Waits for the phase with the given parity; gives up after TC_WAIT_CYCLES or when another
+// role already gave up.  Returns false in that case.
+__device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > TC_WAIT_CYCLES) { *abort_flag = 1; return false; }
+  }
+}
+
+__device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ inline void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ inline void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ inline void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ inline void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ inline void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+               "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr));
+}
+__device__ inline void tc_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+               "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                 "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                 "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+               : "memory");
+}
+__device__ inline void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ inline void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
+// K-major operand: rows of 64 bf16 (128 bytes); the leading offset is unused.
+__device__ inline uint64_t desc_kmajor(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand (V: keys x d, d contiguous): the next 64-element block of d starts
+// TC_HALF_BYTES further, the next group of 8 keys 1024 bytes further.
+__device__ inline uint64_t desc_mnmajor(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(TC_HALF_BYTES >> 4) << 16) | (64ull << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128.
+constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t IDESC_QK = idesc_base;                 // A and B K-major
+constexpr uint32_t IDESC_PV = idesc_base | (1u << 16);    // B MN-major
+
+__device__ inline float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ inline uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kp,
+                         const __grid_constant__ CUtensorMap map_vp, const __grid_constant__ CUtensorMap map_kt,
+                         const __grid_constant__ CUtensorMap map_vt, TcArgs a) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int mpair = blockIdx.x, split = blockIdx.y;
+  const int bh = blockIdx.z, b = bh / a.Hkv, kvh = bh - b * a.Hkv;
+
+  // carve shared memory: tiles need 1024-byte alignment for the 128-byte swizzle
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const uint32_t q_smem = base;
+  const uint32_t k_smem = base + 2 * TC_TILE_BYTES;
+  const uint32_t v_smem = k_smem + TC_STAGES * TC_TILE_BYTES;
+  const uint32_t bars = v_smem + TC_STAGES * TC_TILE_BYTES;
+  unsigned char *gen_base = smem_dyn + (base - smem_u32(smem_dyn));      // generic pointer to `base`
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+
+  const int n = a.n_nodes[b];
+  const int L = a.prefix_len[b];
+  const int rows_total = a.g * a.N;
+  const int rows_valid = a.g * n;
+  int nmt = (rows_total - mpair * 2 * TC_MT + TC_MT - 1) / TC_MT;       // query tiles of this CTA with rows
+  nmt = nmt > 2 ? 2 : nmt;
+
+  const int nP = (L + TC_BN - 1) / TC_BN;
+  const int nT = (a.N + TC_BN - 1) / TC_BN;
+  const int tt = nP + nT;
+  const int tps = (tt + a.splits - 1) / a.splits;
+  const int t_begin = split * tps;
+  const int t_end = min(tt, t_begin + tps);
+  const int nt = max(t_end - t_begin, 0);
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(bar(B_Q), 1);
+    for (int s = 0; s < TC_STAGES; ++s) {
+      mbar_init(bar(B_KFULL + s), 1);
+      mbar_init(bar(B_VFULL + s), 1);
+      mbar_init(bar(B_KEMPTY + s), 1);
+      mbar_init(bar(B_VEMPTY + s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(B_SFULL + i), 1);
+      mbar_init(bar(B_PFULL + i), 128);
+      mbar_init(bar(B_ODONE + i), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 9) {          // this warp owns the tensor-memory allocation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(TC_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem_base;
+  volatile int *abort_flag = &s_abort;
+
+  if (warp == 8) {
+    // ================= producer =================
+    if (lane == 0 && nt > 0) {
+      const int nodes_per_tile = TC_MT / a.g;
+      mbar_expect_tx(bar(B_Q), (uint32_t)nmt * TC_TILE_BYTES);
+      for (int i = 0; i < nmt; ++i)
+        for (int h = 0; h < 2; ++h)
+          tma_load_4d(q_smem + i * TC_TILE_BYTES + h * TC_HALF_BYTES, &map_q, bar(B_Q), h * 64, kvh * a.g,
+                      (mpair * 2 + i) * nodes_per_tile, b);
+      const long long tok0 = a.kv_start[b];
+      bool ok = true;
+      for (int it = 0; it < nt && ok; ++it) {
+        const int s = it % TC_STAGES;
+        const uint32_t par = ((it / TC_STAGES) & 1) ^ 1;
+        const int tg = t_begin + it;
+        ok = mbar_wait(bar(B_KEMPTY + s), par, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar(B_KFULL + s), TC_TILE_BYTES);
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t dst = k_smem + s * TC_TILE_BYTES + h * TC_HALF_BYTES;
+          if (tg < nP) tma_load_3d(dst, &map_kp, bar(B_KFULL + s), h * 64, kvh, (int)(tok0 + (long long)tg * TC_BN));
+          else tma_load_4d(dst, &map_kt, bar(B_KFULL + s), h * 64, kvh, (tg - nP) * TC_BN, b);
+        }
+        ok = mbar_wait(bar(B_VEMPTY + s), par, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar(B_VFULL + s), TC_TILE_BYTES);
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t dst = v_smem + s * TC_TILE_BYTES + h * TC_HALF_BYTES;
+          if (tg < nP) tma_load_3d(dst, &map_vp, bar(B_VFULL + s), h * 64, kvh, (int)(tok0 + (long long)tg * TC_BN));
+          else tma_load_4d(dst, &map_vt, bar(B_VFULL + s), h * 64, kvh, (tg - nP) * TC_BN, b);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // ================= MMA issue =================
+    if (lane == 0 && nt > 0) {
+      bool ok = mbar_wait(bar(B_Q), 0, abort_flag);
+      auto issue_qk = [&](int i, int s) {
+#pragma unroll
+        for (int kk = 0; kk < TC_D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * TC_HALF_BYTES + (kk & 3) * 32;
+          tc_mma_ss(tmem + 256 + 128 * i, desc_kmajor(q_smem + i * TC_TILE_BYTES + off),
+                    desc_kmajor(k_smem + s * TC_TILE_BYTES + off), IDESC_QK, kk > 0 ? 1u : 0u);
+        }
+      };
+      auto issue_pv = [&](int i, int s, bool accumulate) {
+#pragma unroll
+        for (int kk = 0; kk < TC_BN / 16; ++kk)
+          tc_mma_ts(tmem + 128 * i, tmem + 256 + 128 * i + kk * 8, desc_mnmajor(v_smem + s * TC_TILE_BYTES + kk * 2048),
+                    IDESC_PV, (accumulate || kk > 0) ? 1u : 0u);
+      };
+      if (ok) ok = mbar_wait(bar(B_KFULL + 0), 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        for (int i = 0; i < nmt; ++i) {
+          issue_qk(i, 0);
+          tc_commit(bar(B_SFULL + i));
+        }
+        tc_commit(bar(B_KEMPTY + 0));
+      }
+      for (int it = 0; it < nt && ok; ++it) {
+        const int s = it % TC_STAGES;
+        ok = mbar_wait(bar(B_VFULL + s), (it / TC_STAGES) & 1, abort_flag);
+        for (int i = 0; i < nmt && ok; ++i) {
+          ok = mbar_wait(bar(B_PFULL + i), it & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(i, s, it > 0);
+          tc_commit(bar(B_ODONE + i));
+          if (i == nmt - 1) tc_commit(bar(B_VEMPTY + s));
+          if (it + 1 < nt) {
+            const int s2 = (it + 1) % TC_STAGES;
+            if (i == 0) {
+              ok = mbar_wait(bar(B_KFULL + s2), ((it + 1) / TC_STAGES) & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_qk(i, s2);
+            tc_commit(bar(B_SFULL + i));
+            if (i == nmt - 1) tc_commit(bar(B_KEMPTY + s2));
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================= softmax + epilogue: warps 0-3 own query tile 0, warps 4-7 tile 1 =================
+    const int i = warp >> 2;
+    const int quarter = warp & 3;
+    const int r_local = quarter * 32 + lane;
+    const int R = (mpair * 2 + i) * TC_MT + r_local;            // packed query row
+    const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t t_S = t_lane + 256 + 128 * i;
+    const uint32_t t_O = t_lane + 128 * i;
+    const bool row_valid = R < rows_valid;
+    unsigned long long mrow[2] = {0ull, 0ull};
+    if (row_valid)
+      for (int w = 0; w < a.W; ++w) mrow[w] = a.mask[((int64_t)b * a.N + R / a.g) * a.W + w];
+
+    float m_used = -CUDART_INF_F, l_run = 0.f;
+    bool ok = (i < nmt) && nt > 0;
+    for (int it = 0; it < nt && ok; ++it) {
+      const int tg = t_begin + it;
+      const bool tree_tile = tg >= nP;
+      const int kvalid = tree_tile ? min(n - (tg - nP) * TC_BN, TC_BN) : min(L - tg * TC_BN, TC_BN);
+      const int s = it % TC_STAGES;
+      // keys beyond the valid range may hold anything: tile 0's warps clear their V rows so that
+      // a zero probability times stale memory cannot produce a NaN
+      if (i == 0 && kvalid < TC_BN) {
+        ok = mbar_wait(bar(B_VFULL + s), (it / TC_STAGES) & 1, abort_flag);
+        if (!ok) break;
+        const int zr = max(kvalid, 0) + r_local;
+        if (zr < TC_BN) {
+          uint4 *p0 = reinterpret_cast<uint4 *>(gen_base + (2 + TC_STAGES) * TC_TILE_BYTES + s * TC_TILE_BYTES + zr * 128);
+          uint4 *p1 = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(p0) + TC_HALF_BYTES);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) { p0[c] = make_uint4(0, 0, 0, 0); p1[c] = make_uint4(0, 0, 0, 0); }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      }
+      ok = mbar_wait(bar(B_SFULL + i), it & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+
+      const bool masked = tree_tile || kvalid < TC_BN;
+      const unsigned long long vis0 = tree_tile ? mrow[0] : ~0ull, vis1 = tree_tile ? mrow[1] : ~0ull;
+      // keys c of this tile the row may see: c < kvalid and (tree tile) ancestor bit c
+      unsigned long long see0 = vis0, see1 = vis1;
+      if (kvalid < 64) { see0 &= kvalid <= 0 ? 0ull : (~0ull >> (64 - kvalid)); see1 = 0ull; }
+      else if (kvalid < 128) see1 &= kvalid == 64 ? 0ull : (~0ull >> (128 - kvalid));
+      if (tree_tile && (tg - nP) > 0) { see0 = 0ull; see1 = 0ull; }     // N <= 128: there is one tree tile
+
+      // ---- pass 1: row maximum ----
+      float mx = -CUDART_INF_F;
+#pragma unroll
+      for (int c0 = 0; c0 < TC_BN; c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(t_S + c0, r);
+        tc_wait_ld();
+        if (masked) {
+          const uint32_t bits = (uint32_t)((c0 < 64 ? see0 : see1) >> (c0 & 63));
+#pragma unroll
+          for (int c = 0; c < 32; ++c) mx = fmaxf(mx, ((bits >> c) & 1u) ? __uint_as_float(r[c]) : -CUDART_INF_F);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(r[c]));
+        }
+      }
+      const float mx_x = mx * a.scale_log2;
+      float alpha = 1.f;
+      if (m_used == -CUDART_INF_F) m_used = mx_x;
+      else if (mx_x > m_used + TC_RESCALE_GAP) {
+        alpha = fast_exp2(m_used - mx_x);
+        l_run *= alpha;
+        m_used = mx_x;
+      }
+      const float m_eff = (m_used == -CUDART_INF_F) ? 0.f : m_used;
+
+      // ---- pass 2: P = exp2(S * scale - max) as bf16 over S; row sum ----
+      float sum = 0.f;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int c0 = half * 64 + q * 32;
+          uint32_t r[32];
+          tc_ld32(t_S + c0, r);
+          tc_wait_ld();
+          const uint32_t bits = masked ? (uint32_t)((c0 < 64 ? see0 : see1) >> (c0 & 63)) : 0xFFFFFFFFu;
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            float p0 = fast_exp2(fmaf(__uint_as_float(r[c]), a.scale_log2, -m_eff));
+            float p1 = fast_exp2(fmaf(__uint_as_float(r[c + 1]), a.scale_log2, -m_eff));
+            if (!((bits >> c) & 1u)) p0 = 0.f;
+            if (!((bits >> (c + 1)) & 1u)) p1 = 0.f;
+            sum += p0 + p1;
+            pk[q * 16 + (c >> 1)] = pack_bf16x2(p0, p1);
+          }
+        }
+        tc_st32(t_S + half * 32, pk);
+      }
+      l_run += sum;
+
+      // ---- rare: the reference maximum moved, rescale the accumulator of this row's warp ----
+      if (it > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+        ok = mbar_wait(bar(B_ODONE + i), (it - 1) & 1, abort_flag);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < TC_D; c0 += 32) {
+            uint32_t r[32];
+            tc_ld32(t_O + c0, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+            tc_st32(t_O + c0, r);
+          }
+        }
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(B_PFULL + i));
+    }
+
+    // ---- epilogue: O / l (or the partial result of this key range) ----
+    if (ok) ok = mbar_wait(bar(B_ODONE + i), (nt - 1) & 1, abort_flag);
+    if (ok && R < rows_total) {
+      tc_fence_after();
+      const int node = R / a.g, qh = R - node * a.g;
+      if (a.splits == 1) {
+        const bool live = row_valid && l_run > 0.f;
+        const float inv = live ? 1.f / l_run : 0.f;
+        __nv_bfloat16 *op = a.out + (((int64_t)b * a.N + node) * a.Hq + kvh * a.g + qh) * TC_D;
+#pragma unroll
+        for (int c0 = 0; c0 < TC_D; c0 += 32) {
+          uint32_t r[32];
+          tc_ld32(t_O + c0, r);
+          tc_wait_ld();
+          uint32_t o[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            o[c] = live ? pack_bf16x2(__uint_as_float(r[2 * c]) * inv, __uint_as_float(r[2 * c + 1]) * inv) : 0u;
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+        }
+      } else if (row_valid) {
+        const int mpad = a.m_blocks * TC_MT;
+        const int64_t prow = ((int64_t)bh * a.splits + split) * mpad + R;
+        float *op = a.part_o + prow * TC_D;
+#pragma unroll
+        for (int c0 = 0; c0 < TC_D; c0 += 32) {
+          uint32_t r[32];
+          tc_ld32(t_O + c0, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+        }
+        a.part_ml[prow] = make_float2(m_used, l_run);
+      }
+    } else if (nt == 0 && i < nmt && R < rows_total) {
+      // an empty key range (more splits than tiles): contribute nothing
+      if (a.splits == 1) {
+        const int node = R / a.g, qh = R - node * a.g;
+        uint4 *op = reinterpret_cast<uint4 *>(a.out + (((int64_t)b * a.N + node) * a.Hq + kvh * a.g + qh) * TC_D);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) op[c] = make_uint4(0, 0, 0, 0);
+      } else if (row_valid) {
+        const int mpad = a.m_blocks * TC_MT;
+        a.part_ml[((int64_t)bh * a.splits + split) * mpad + R] = make_float2(-CUDART_INF_F, 0.f);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS) : "memory");
+  }
+  if (tid == 0 && s_abort) atomicOr(a.status, STATUS_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+bool encode_bf16(CUtensorMap *m, const void *ptr, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes,
+                 const cuuint32_t *box) {
+  const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(ptr), dims,
+                        strides_bytes, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) std::fprintf(stderr, "talon: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool attention_tc_supported(const talon_ctx *c, int64_t stride_t, int64_t stride_h, float sm_scale) {
+  const int g = c->p.n_q_heads / c->p.n_kv_heads;
+  if (c->p.head_dim != 128 || c->p.budget > 128) return false;
+  if (g < 1 || g > 128 || (128 % g) != 0) return false;
+  if (!(sm_scale > 0.f)) return false;                     // the lazy maximum assumes a positive scale
+  if (stride_t < 128 || stride_h < 1) return false;
+  return encode_fn() != nullptr;
+}
+
+talon_status attention_tc_setup() {
+  return cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM) ==
+                 cudaSuccess ? TALON_OK : TALON_ERR_CUDA;
+}
+
+talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
+                                 const void *kt, const void *vt, const int64_t *kv_start, int64_t stride_t,
+                                 int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
+                                 int splits, int m_blocks, cudaStream_t st) {
+  const int N = c->p.budget, Hq = c->p.n_q_heads, Hkv = c->p.n_kv_heads, g = Hq / Hkv, B = c->B;
+  CUtensorMap mq, mkp, mvp, mkt, mvt;
+  {
+    const cuuint64_t dims[4] = {128, (cuuint64_t)Hq, (cuuint64_t)N, (cuuint64_t)B};
+    const cuuint64_t str[3] = {256, (cuuint64_t)Hq * 256, (cuuint64_t)N * Hq * 256};
+    const cuuint32_t box[4] = {64, (cuuint32_t)g, (cuuint32_t)(128 / g), 1};
+    if (!encode_bf16(&mq, q, 4, dims, str, box)) return TALON_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[3] = {128, (cuuint64_t)Hkv, (cuuint64_t)(kv_tokens > 0 ? kv_tokens : 1)};
+    const cuuint64_t str[2] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2};
+    const cuuint32_t box[3] = {64, 1, TC_BN};
+    if (!encode_bf16(&mkp, kp, 3, dims, str, box) || !encode_bf16(&mvp, vp, 3, dims, str, box)) return TALON_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[4] = {128, (cuuint64_t)Hkv, (cuuint64_t)N, (cuuint64_t)B};
+    const cuuint64_t str[3] = {256, (cuuint64_t)Hkv * 256, (cuuint64_t)N * Hkv * 256};
+    const cuuint32_t box[4] = {64, 1, TC_BN, 1};
+    if (!encode_bf16(&mkt, kt, 4, dims, str, box) || !encode_bf16(&mvt, vt, 4, dims, str, box)) return TALON_ERR_CUDA;
+  }
+  TcArgs a;
+  a.kv_start = kv_start; a.prefix_len = c->d_prefix_len; a.n_nodes = t->n_nodes;
+  a.mask = (const unsigned long long *)t->mask;
+  a.B = B; a.N = N; a.W = c->W; a.Hq = Hq; a.Hkv = Hkv; a.g = g;
+  a.scale_log2 = sm_scale * 1.4426950408889634f;
+  a.splits = splits; a.m_blocks = m_blocks;
+  a.out = (__nv_bfloat16 *)out; a.part_o = c->d_attn_o; a.part_ml = c->d_attn_ml; a.status = c->d_status;
+  (void)max_prefix_len;
+  dim3 grid((m_blocks + 1) / 2, splits, B * Hkv);
+  {
+    LaunchTimer lt(c, TALON_K_ATTENTION, st);
+    tree_attention_tc_kernel<<<grid, TC_THREADS, TC_SMEM, st>>>(mq, mkp, mvp, mkt, mvt, a);
+  }
+  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+  c->launches += 1;
+  return TALON_OK;
+}
+
+}  // namespace talon

@@ -31,7 +31,7 @@ struct FusedArgs {
   int rows_per_seq, layout;
   talon_tree t;
   int lo_stride;
-  int B, N, W, V, d, k, key_stride, target_items, max_splits;
+  int B, N, W, V, d, k, key_stride, target_items, max_splits, items_cap;
   int root_topk, init_layers;
   double log_mu;
   u64 *part_keys;          // [items, key_stride]  per-chunk top-k, descending
@@ -174,6 +174,40 @@ __device__ inline u64 f64_ord(double x) {
 __device__ inline double f64_unord(u64 o) {
   const u64 b = (o >> 63) ? (o & 0x7FFFFFFFFFFFFFFFull) : ~o;
   return __longlong_as_double((long long)b);
+}
+
+// Chunks per row for this layer.  Every CTA of the grid is resident, so a layer takes
+// ceil(items / grid) rounds of one chunk each: the cost of a candidate split count is
+// rounds x (chunk length + a fixed per-chunk overhead), in units of 1024 elements.  Lane l
+// scores the counts l + 1 and l + 33; the warp keeps the cheapest (the smaller count on ties).
+__device__ inline LayerGeom balanced_geom(int total_rows, int vocab, int grid, int max_splits, int items_cap) {
+  const int lane = threadIdx.x & 31;
+  unsigned best = 0xFFFFFFFFu;               // cost << 8 | splits
+  if (total_rows > 0) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int sp = lane + 1 + 32 * i;
+      if (sp > max_splits) continue;
+      int len = (vocab + sp - 1) / sp;
+      len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
+      if (len < EXP_TILE && sp > 1) continue;
+      const int eff = (vocab + len - 1) / len;
+      if (sp > 1 && (long long)total_rows * eff > items_cap) continue;   // workspace holds items_cap chunk results
+      const int rounds = (total_rows * eff + grid - 1) / grid;
+      const unsigned cost = (unsigned)rounds * (unsigned)(len / EXP_CHUNK_ALIGN + 8);
+      const unsigned packed = (min(cost, 0xFFFFFFu) << 8) | (unsigned)eff;
+      best = min(best, packed);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
+  LayerGeom g;
+  g.total_rows = total_rows;
+  g.splits = total_rows > 0 ? (int)(best & 0xFFu) : 1;
+  int len = (vocab + g.splits - 1) / g.splits;
+  g.chunk_len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
+  g.splits = (vocab + g.chunk_len - 1) / g.chunk_len;
+  return g;
 }
 
 // Where a packed frontier row lives: sequence, index inside that sequence's frontier, tree
@@ -485,7 +519,7 @@ expand_fused_kernel(FusedArgs a) {
         if (s_base[b + 1] == s_base[b]) a.t.layer_off[b * a.lo_stride + a.d + 2] = a.t.n_nodes[b];
   }
   if (tid == 0) s_pool_n = 0;
-  const LayerGeom g = make_geom(fr.total, a.V, a.target_items, a.max_splits, EXP_TILE);
+  const LayerGeom g = balanced_geom(fr.total, a.V, a.target_items, a.max_splits, a.items_cap);
   const int n_items = fr.total * g.splits;
   __syncthreads();
 
@@ -712,7 +746,8 @@ talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float 
   int grid = c->fused_grid;
   if (max_items < grid) grid = (int)max_items;
   if (grid < 1) grid = 1;
-  a.target_items = c->fused_grid;
+  a.target_items = grid;
+  a.items_cap = c->items_cap;
   a.root_topk = c->p.root_topk; a.init_layers = c->p.init_layers; a.log_mu = c->log_mu;
   a.part_keys = c->d_part_keys; a.part_ms = c->d_part_ms; a.seq_count = c->d_seq_count; a.status = c->d_status;
   {

@@ -149,8 +149,13 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
 talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cudaStream_t st);
 talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp,
                               const void *vp, const void *kt, const void *vt,
-                              const int64_t *kv_start, int64_t stride_t, int64_t stride_h,
+                              const int64_t *kv_start, int64_t kv_tokens, int64_t stride_t, int64_t stride_h,
                               int max_prefix_len, float sm_scale, void *out, cudaStream_t st);
+bool attention_tc_supported(const talon_ctx *c, int64_t stride_t, int64_t stride_h, float sm_scale);
+talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
+                                 const void *kt, const void *vt, const int64_t *kv_start, int64_t stride_t,
+                                 int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
+                                 int splits, int m_blocks, cudaStream_t st);
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                            int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st);

@@ -45,11 +45,11 @@ _lib.talon_reset.argtypes = [_vp, _TP, _vp, _vp, _i32, _vp]
 _lib.talon_expand_layer.argtypes = [_vp, _TP, _vp, _i64, _i32, _i32, _vp]
 _lib.talon_layers_run.argtypes = [_vp]
 _lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
-_lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i32, _f32, _vp, _vp]
+_lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_poll_status.argtypes = [_vp, _vp]
 _lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
-_lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i32, _f32, _vp,
+_lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i64, _i32, _f32, _vp,
                             _vp, _i64] + [_vp] * 5)
 _lib.talon_timing_enable.argtypes = [_vp, _i32, C.c_uint32]
 _lib.talon_timing_read.argtypes = [_vp, _vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -166,11 +166,11 @@ class Talon:
         _check(_lib.talon_build_tree(self._ctx, C.byref(ts), _ptr(dense_mask), _stream(self.device)),
                "talon_build_tree")
 
-    def tree_attention(self, tree: Tree, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_stride_t,
+    def tree_attention(self, tree: Tree, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_tokens, kv_stride_t,
                        kv_stride_h, max_prefix_len, sm_scale, out):
         ts = tree.struct()
         _check(_lib.talon_tree_attention(self._ctx, C.byref(ts), _ptr(q), _ptr(k_prefix), _ptr(v_prefix),
-                                         _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_stride_t, kv_stride_h,
+                                         _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_tokens, kv_stride_t, kv_stride_h,
                                          max_prefix_len, sm_scale, _ptr(out), _stream(self.device)),
                "talon_tree_attention")
 
@@ -190,14 +190,14 @@ class Talon:
         return _lib.talon_launch_count(self._ctx)
 
     def step(self, tree: Tree, root_tok, prefix_len, draft_logits, n_layers, q, k_prefix, v_prefix, k_tree, v_tree,
-             kv_start, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out, target_logits, target_tok,
+             kv_start, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out, target_logits, target_tok,
              accept_len, accept_nodes, bonus_tok):
         """``talon_step``: the whole draft-and-verify step on device-resident inputs, one library call."""
         ts = tree.struct()
         _check(_lib.talon_step(self._ctx, C.byref(ts), root_tok.shape[0], _ptr(root_tok), _ptr(prefix_len),
                                _ptr(draft_logits), draft_logits.stride(-2), n_layers, _ptr(q), _ptr(k_prefix),
-                               _ptr(v_prefix), _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_stride_t, kv_stride_h,
-                               max_prefix_len, sm_scale, _ptr(out), _ptr(target_logits), target_logits.stride(-2),
+                               _ptr(v_prefix), _ptr(k_tree), _ptr(v_tree), _ptr(kv_start), kv_tokens, kv_stride_t,
+                               kv_stride_h, max_prefix_len, sm_scale, _ptr(out), _ptr(target_logits), target_logits.stride(-2),
                                _ptr(target_tok), _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok),
                                _stream(self.device)), "talon_step")
 

@@ -151,7 +151,7 @@ def run_step(talon: Talon, wl: Workload, sm_scale: Optional[float] = None, expan
         talon.expand_layer(wl.tree, wl.draft)
     talon.build_tree(wl.tree)
     talon.tree_attention(wl.tree, wl.q, wl.k_prefix, wl.v_prefix, wl.k_tree, wl.v_tree, wl.kv_start,
-                         cfg.n_kv_heads * cfg.head_dim, cfg.head_dim, wl.max_prefix_len, sm_scale, wl.out)
+                         wl.k_prefix.shape[0], cfg.n_kv_heads * cfg.head_dim, cfg.head_dim, wl.max_prefix_len, sm_scale, wl.out)
     talon.accept(wl.tree, wl.target, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok)
 
 
@@ -161,6 +161,7 @@ def run_step_fused(talon: Talon, wl: Workload, sm_scale: Optional[float] = None,
     if sm_scale is None:
         sm_scale = 1.0 / float(np.sqrt(cfg.head_dim))
     talon.step(wl.tree, wl.root_tok, wl.prefix_len, wl.draft, cfg.max_depth if n_layers is None else n_layers,
-               wl.q, wl.k_prefix, wl.v_prefix, wl.k_tree, wl.v_tree, wl.kv_start, cfg.n_kv_heads * cfg.head_dim,
+               wl.q, wl.k_prefix, wl.v_prefix, wl.k_tree, wl.v_tree, wl.kv_start, wl.k_prefix.shape[0],
+               cfg.n_kv_heads * cfg.head_dim,
                cfg.head_dim, wl.max_prefix_len, sm_scale, wl.out, wl.target, wl.target_tok, wl.accept_len,
                wl.accept_nodes, wl.bonus_tok)
