@@ -346,7 +346,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       // keys beyond the valid range may hold anything: tile 0's warps clear their V rows so that
       // a zero probability times stale memory cannot produce a NaN
       if (i == 0 && kvalid < TC_BN) {
-        ok = mbar_wait(bar(B_VFULL + s), (it / TC_STAGES) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(B_VFULL + s), (it / TC_STAGES) & 1, abort_flag));
         if (!ok) break;
         const int zr = max(kvalid, 0) + r_local;
         if (zr < TC_BN) {
@@ -357,7 +357,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       }
-      ok = mbar_wait(bar(B_SFULL + i), it & 1, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(B_SFULL + i), it & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
 
@@ -423,7 +423,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
       // ---- rare: the reference maximum moved, rescale the accumulator of this row's warp ----
       if (it > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-        ok = mbar_wait(bar(B_ODONE + i), (it - 1) & 1, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(B_ODONE + i), (it - 1) & 1, abort_flag));
         if (ok) {
           tc_fence_after();
 #pragma unroll
@@ -443,10 +443,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     }
 
     // ---- epilogue: O / l (or the partial result of this key range) ----
-    if (ok) ok = mbar_wait(bar(B_ODONE + i), (nt - 1) & 1, abort_flag);
-    if (ok && R < rows_total) {
+    // tcgen05.ld is a warp-wide instruction: every lane of a warp that holds any row takes part
+    // in the loads, and only the stores are per lane.
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(B_ODONE + i), (nt - 1) & 1, abort_flag));
+    const bool in_range = R < rows_total;
+    if (ok && __any_sync(0xFFFFFFFFu, in_range)) {
       tc_fence_after();
-      const int node = R / a.g, qh = R - node * a.g;
+      const int node = in_range ? R / a.g : 0, qh = in_range ? R - node * a.g : 0;
       if (a.splits == 1) {
         const bool live = row_valid && l_run > 0.f;
         const float inv = live ? 1.f / l_run : 0.f;
@@ -460,24 +463,28 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
           for (int c = 0; c < 16; ++c)
             o[c] = live ? pack_bf16x2(__uint_as_float(r[2 * c]) * inv, __uint_as_float(r[2 * c + 1]) * inv) : 0u;
+          if (in_range) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
-            reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+            for (int c = 0; c < 4; ++c)
+              reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+          }
         }
-      } else if (row_valid) {
+      } else {
         const int mpad = a.m_blocks * TC_MT;
-        const int64_t prow = ((int64_t)bh * a.splits + split) * mpad + R;
+        const int64_t prow = ((int64_t)bh * a.splits + split) * mpad + (in_range ? R : 0);
         float *op = a.part_o + prow * TC_D;
 #pragma unroll
         for (int c0 = 0; c0 < TC_D; c0 += 32) {
           uint32_t r[32];
           tc_ld32(t_O + c0, r);
           tc_wait_ld();
+          if (row_valid) {
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
-            reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+            for (int c = 0; c < 8; ++c)
+              reinterpret_cast<uint4 *>(op + c0)[c] = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+          }
         }
-        a.part_ml[prow] = make_float2(m_used, l_run);
+        if (row_valid) a.part_ml[prow] = make_float2(m_used, l_run);
       }
     } else if (nt == 0 && i < nmt && R < rows_total) {
       // an empty key range (more splits than tiles): contribute nothing
