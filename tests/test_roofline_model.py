@@ -1,0 +1,31 @@
+"""The algorithmic-work model that the benchmark's roofline figures use (host logic only)."""
+from paper_2601_07353_b200 import roofline, synth
+
+
+def test_expanded_rows_counts_frontiers_that_still_have_budget():
+    # budget 7: layers of 1, 2, 2, 2 nodes -> frontiers of layers 0..2 are expanded (1 + 2 + 2 rows)
+    assert roofline.expanded_rows([0, 1, 3, 5, 7, 7, 7], 7, 6) == 5
+    # depth stop: only the layers that were enqueued count
+    assert roofline.expanded_rows([0, 1, 3, 5, 7, 7, 7], 7, 2) == 3
+    # a tree that stays below its budget expands its last frontier too, then meets an empty layer
+    assert roofline.expanded_rows([0, 1, 2, 3, 3, 3], 10, 5) == 3
+
+
+def test_bytes_match_the_stated_per_unit_figures():
+    cfg = synth.CONFIGS["llama8b"]
+    assert roofline.expand_bytes(3, cfg.vocab) == 3 * 4 * cfg.vocab
+    assert roofline.argmax_bytes(60, cfg.vocab) == 60 * 4 * cfg.vocab
+    b = roofline.attention_bytes(2048, 60, 32, 8, 128, 60)
+    assert b == 2 * 2 * 128 * 8 * (2048 + 60) + 2 * 2 * 60 * 32 * 128 + 8 * 1 * 60
+    f = roofline.attention_flops(2048, 60, 32, 128)
+    assert f == 4 * 128 * 32 * 60 * 2108
+    # arithmetic intensity is g * N flop per KV byte up to the Q/O and mask terms
+    assert abs(f / (2 * 2 * 128 * 8 * 2108) - 4 * 60) < 1e-9
+
+
+def test_peaks_fall_back_when_the_file_is_missing(tmp_path):
+    p = roofline.load_peaks(str(tmp_path))
+    assert p["source"] == "fallback" and p["hbm_gbs"] == roofline.FALLBACK_HBM_GBS
+    (tmp_path / "MEASURED_PEAKS.json").write_text('{"hbm_gbs": 6000.0, "bf16_tflops": 1500.0}')
+    p = roofline.load_peaks(str(tmp_path))
+    assert p["source"] == "measured" and p["hbm_gbs"] == 6000.0 and p["bf16_tflops_sustained"] == 1500.0
