@@ -1,18 +1,24 @@
 // Adaptive draft-tree expansion (Algorithm 2 of the paper; Eq. 2-5) as ONE kernel per layer,
 // for per-parent candidate caps k <= 32 (the usual case: the paper's K is 10).
 //
-// Streaming phase.  The frontier's fp32 logit rows are cut into chunks, one CTA per chunk at a
-// time.  In a single read of its chunk a CTA produces the chunk's share of the softmax
-// normaliser of Eq. 3 (running maximum and sum of exponentials) and the chunk's k largest
-// logits with their token ids.  Each warp keeps a sorted list of its best k keys across its 32
-// lanes plus a small queue of elements that passed the current threshold; a full queue is
-// folded into the list with a bitonic sort and merge, which also raises the threshold.
+// Streaming phase.  The frontier's fp32 logit rows are cut into equal chunks, one CTA per chunk
+// at a time.  In a single read of its chunk a CTA produces the chunk's share of the softmax
+// normaliser of Eq. 3 (maximum and sum of exponentials) and the chunk's k largest logits with
+// their token ids.
+//   * A chunk of at most 4096 elements sits in registers (16 per thread).  The smallest of the
+//     256/G maxima of G-lane groups bounds the chunk's k-th largest element from below (the
+//     groups hold 256/G >= k different elements that large), so only elements at or above it
+//     go to a shared pool, which is then ranked by counting.
+//   * A longer chunk is streamed tile by tile; each warp keeps a sorted list of its best k
+//     keys across its lanes plus a queue of elements that passed the current threshold, and a
+//     full queue is folded into the list with a bitonic sort and merge.
 //
 // Selection phase.  The CTA that finishes the last chunk of a sequence merges that sequence's
 // chunk results into per-row top-k lists and log-sum-exps, scores the pooled candidates with
 // log p(u) = log p(v) + log P(w | v) (Eq. 2-3), applies Top-K (Eq. 5) or the confidence gate
 // p(u) >= mu * max p (Eq. 4), truncates to the remaining budget, and appends the survivors with
 // parent links, depths, scores and ancestor-mask rows.  Nothing returns to the host in between.
+#include <cuda/atomic>
 #include <math_constants.h>
 
 #include "talon_internal.cuh"
@@ -178,25 +184,22 @@ __device__ inline double f64_unord(u64 o) {
 
 // Chunks per row for this layer.  Every CTA of the grid is resident, so a layer takes
 // ceil(items / grid) rounds of one chunk each: the cost of a candidate split count is
-// rounds x (chunk length + a fixed per-chunk overhead), in units of 1024 elements.  Lane l
-// scores the counts l + 1 and l + 33; the warp keeps the cheapest (the smaller count on ties).
+// rounds x (tiles per chunk + a fixed per-chunk overhead of about two tiles).  Chunks of one
+// row are equal up to rounding to 4 elements (rows are 16-byte aligned), and a split row keeps
+// at least 1024 elements per chunk so that every warp of a CTA holds some.  Lane l scores the
+// split count l + 1; the warp keeps the cheapest (the smaller count on ties).
 __device__ inline LayerGeom balanced_geom(int total_rows, int vocab, int grid, int max_splits, int items_cap) {
   const int lane = threadIdx.x & 31;
   unsigned best = 0xFFFFFFFFu;               // cost << 8 | splits
   if (total_rows > 0) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int sp = lane + 1 + 32 * i;
-      if (sp > max_splits) continue;
-      int len = (vocab + sp - 1) / sp;
-      len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
-      if (len < EXP_TILE && sp > 1) continue;
-      const int eff = (vocab + len - 1) / len;
-      if (sp > 1 && (long long)total_rows * eff > items_cap) continue;   // workspace holds items_cap chunk results
+    const int sp = lane + 1;
+    int len = (((vocab + sp - 1) / sp) + 3) & ~3;
+    const int eff = (vocab + len - 1) / len;
+    const bool fits = sp == 1 || (sp <= max_splits && len >= 1024 && (long long)total_rows * eff <= items_cap);
+    if (fits) {
       const int rounds = (total_rows * eff + grid - 1) / grid;
-      const unsigned cost = (unsigned)rounds * (unsigned)(len / EXP_CHUNK_ALIGN + 8);
-      const unsigned packed = (min(cost, 0xFFFFFFu) << 8) | (unsigned)eff;
-      best = min(best, packed);
+      const unsigned cost = (unsigned)rounds * (unsigned)(2 * ((len + EXP_TILE - 1) / EXP_TILE) + 4);
+      best = (min(cost, 0xFFFFFFu) << 8) | (unsigned)eff;
     }
   }
 #pragma unroll
@@ -204,8 +207,7 @@ __device__ inline LayerGeom balanced_geom(int total_rows, int vocab, int grid, i
   LayerGeom g;
   g.total_rows = total_rows;
   g.splits = total_rows > 0 ? (int)(best & 0xFFu) : 1;
-  int len = (vocab + g.splits - 1) / g.splits;
-  g.chunk_len = ((len + EXP_CHUNK_ALIGN - 1) / EXP_CHUNK_ALIGN) * EXP_CHUNK_ALIGN;
+  g.chunk_len = (((vocab + g.splits - 1) / g.splits) + 3) & ~3;
   g.splits = (vocab + g.chunk_len - 1) / g.chunk_len;
   return g;
 }
@@ -247,7 +249,7 @@ __device__ inline RowLoc locate_row(const FusedArgs &a, const Frontier &fr, int 
 
 // Shared-memory carve-up of the selection phase.
 struct TailSmem {
-  u64 *stage;        // [EXP_WARPS][FX_STAGE]  chunk lists of the row a warp is merging
+  u64 *stage;        // [EXP_WARPS][32 k + FX_SURV]  chunk lists of the row a warp is merging, survivors
   u64 *row_keys;     // [N-1][k]               per-row top-k keys, descending
   double *score;     // [N-1][k]               log p(u) of each pooled candidate
   double *row_t;     // [N-1]                  sum of exponentials, then the row's log-sum-exp
@@ -269,82 +271,83 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
   const size_t nb = (size_t)b * a.N;
   if (tid == 0) { *s_anchor = 0ull; *s_cnt = 0; *s_bad = 0; }
 
-  // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys ----
+  // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys.
+  // One warp per row, one lane per chunk (S <= 32). ----
+  const int stage_words = 32 * k + FX_SURV;
   for (int j = warp; j < F; j += EXP_WARPS) {
     const size_t item0 = (size_t)(row0 + j) * S;
-    // everything this row needs from global memory, issued together
-    float2 ms[2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int c = lane + 32 * i;
-      ms[i] = (c < S) ? __ldcg(a.part_ms + item0 + c) : make_float2(-CUDART_INF_F, 0.f);
-    }
-    u64 *st = sm.stage + warp * FX_STAGE;
+    u64 *st = sm.stage + warp * stage_words;       // st[i * 32 + c] = i-th best key of chunk c
+    u64 *sv = st + 32 * k;                         // keys that reach the bound
     u64 *rk = sm.row_keys + (size_t)j * k;
-    const int nk = S * ks;                  // padding slots (p >= k) always hold zero
+    // everything this row needs from global memory, issued together
+    const float2 ms = (lane < S) ? __ldcg(a.part_ms + item0 + lane) : make_float2(-CUDART_INF_F, 0.f);
     if (S == 1) {
       if (lane < k) rk[lane] = __ldcg(a.part_keys + item0 * ks + lane);
-    } else {
-      for (int idx = lane; idx < nk; idx += 32) st[idx] = __ldcg(a.part_keys + item0 * ks + idx);
+    } else if (lane < S) {
+      const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(a.part_keys + (item0 + lane) * ks);
+      for (int i2 = 0; i2 < ks / 2; ++i2) {        // slots k..ks-1 of a list always hold zero
+        const ulonglong2 x = __ldcg(src + i2);
+        if (2 * i2 < k) st[(2 * i2) * 32 + lane] = x.x;
+        if (2 * i2 + 1 < k) st[(2 * i2 + 1) * 32 + lane] = x.y;
+      }
     }
     if (lane == 0) sm.row_ps[j] = a.t.score[nb + lo + j];
     if (lane < a.W) sm.row_mask[j * a.W + lane] = a.t.mask[(nb + lo + j) * a.W + lane];
 
-    float mx = fmaxf(ms[0].x, ms[1].x);
+    float mx = ms.x;
 #pragma unroll
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
     double t = 0.0;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      if (ms[i].y != ms[i].y) t += (double)ms[i].y;                       // NaN or +inf logit in the chunk
-      else if (ms[i].x > -CUDART_INF_F) t += (double)ms[i].y * (double)exp2f((ms[i].x - mx) * LOG2E_F);
-    }
+    if (ms.y != ms.y) t = (double)ms.y;                                   // NaN or +inf logit in the chunk
+    else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
 #pragma unroll
     for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
     if (lane == 0) { sm.row_m[j] = mx; sm.row_t[j] = t; }
     if (S == 1) continue;
 
     if (lane < k) rk[lane] = 0ull;
-    __syncwarp();
     // Two lower bounds of the row's k-th best key: the best k-th key of any one chunk, and the
     // k-th best of the chunk heads (k different chunks each hold a key at least that large).
-    u64 tau = 0ull;
-    for (int c = lane; c < S; c += 32) {
-      tau = umax64(tau, st[c * ks + k - 1]);
-      if (S >= k) {
-        const u64 h = st[c * ks];
-        int cnt = 0;
-        for (int o = 0; o < S; ++o) cnt += (st[o * ks] > h) ? 1 : 0;
-        if (cnt == k - 1) tau = umax64(tau, h);
-      }
+    const u64 head = lane < S ? st[lane] : 0ull;
+    u64 tau = lane < S ? st[(k - 1) * 32 + lane] : 0ull;
+    if (S >= k) {
+      int cnt = 0;
+#pragma unroll 8
+      for (int o = 0; o < 32; ++o) cnt += (shfl_u64(head, o) > head) ? 1 : 0;
+      if (cnt == k - 1) tau = umax64(tau, head);
     }
     tau = warp_max_u64(tau);
-    // compact the keys that reach the bound to the front of the staging area
-    int mine = 0;
-    for (int idx = lane; idx < nk; idx += 32) {
-      const u64 key = st[idx];
-      mine += (key != 0ull && key >= tau) ? 1 : 0;
-    }
-    int inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(FULL, inc, o);
-      if (lane >= o) inc += v;
-    }
-    const int ns = __shfl_sync(FULL, inc, 31);
-    u64 *sv = st + nk;                       // survivors go behind the lists (nk <= FX_STAGE / 2)
-    int pos = inc - mine;
-    for (int idx = lane; idx < nk; idx += 32) {
-      const u64 key = st[idx];
-      if (key != 0ull && key >= tau) sv[pos++] = key;
+    // keys that reach the bound: lists are sorted, so the scan over list positions stops at the
+    // first position where no chunk has one
+    int ns = 0;
+    for (int i = 0; i < k; ++i) {
+      const u64 key = lane < S ? st[i * 32 + lane] : 0ull;
+      const bool ok = key != 0ull && key >= tau;
+      const unsigned mk = __ballot_sync(FULL, ok);
+      if (mk == 0u) break;
+      const int pos = ns + __popc(mk & ((1u << lane) - 1u));
+      if (ok && pos < FX_SURV) sv[pos] = key;
+      ns += __popc(mk);
     }
     __syncwarp();
-    // rank by counting (keys are unique)
-    for (int i = lane; i < ns; i += 32) {
-      const u64 key = sv[i];
-      int r = 0;
-      for (int o = 0; o < ns; ++o) r += (sv[o] > key) ? 1 : 0;
-      if (r < k) rk[r] = key;
+    if (ns <= FX_SURV) {
+      // rank by counting (keys are unique)
+      for (int i = lane; i < ns; i += 32) {
+        const u64 key = sv[i];
+        int r = 0;
+        for (int o = 0; o < ns; ++o) r += (sv[o] > key) ? 1 : 0;
+        if (r < k) rk[r] = key;
+      }
+    } else {
+      // many keys at the bound (equal logits): pop the largest head k times
+      int p = 0;
+      for (int r = 0; r < k; ++r) {
+        const u64 cand = (lane < S && p < k) ? st[p * 32 + lane] : 0ull;
+        const u64 best = warp_max_u64(cand);
+        if (best == 0ull) break;
+        if (cand == best) ++p;
+        if (lane == 0) rk[r] = best;
+      }
     }
     __syncwarp();
   }
@@ -475,14 +478,118 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
   }
 }
 
+// Per-warp state of the streamed top-k: a sorted list across the lanes (once something was
+// folded), a queue in shared memory, and the threshold an element has to reach.
+struct WarpTopk {
+  u64 list;
+  bool folded, first;
+  int qn;
+  float thr0, thr_f;
+};
+
+// One tile (16 elements per thread, already in registers) through the warp's threshold queue.
+// bm is the thread's maximum over the tile.
+__device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC], float bm, int base, int end, int k,
+                                          u64 *queue, WarpTopk &w) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (w.first) {
+    w.first = false;
+    // k lane maxima are k distinct elements, so the k-th largest lane maximum is a lower
+    // bound of this warp's k-th largest element: nothing below it needs to be looked at.
+    int rank = 0;
+#pragma unroll
+    for (int l = 0; l < 32; ++l) {
+      const float o = __shfl_sync(FULL, bm, l);
+      rank += (o > bm) || (o == bm && l < lane);
+    }
+    const unsigned pick = __ballot_sync(FULL, rank == k - 1);
+    if (pick) w.thr0 = __shfl_sync(FULL, bm, __ffs(pick) - 1);
+    w.thr_f = w.thr0;
+  }
+  int mine = 0;
+#pragma unroll
+  for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+    for (int e = 0; e < EXP_VEC; ++e)
+      mine += (v[u][e] >= w.thr_f && base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
+  if (!__any_sync(FULL, mine > 0)) return;
+  int inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(FULL, inc, o);
+    if (lane >= o) inc += t;
+  }
+  const int total = __shfl_sync(FULL, inc, 31);
+  if (total <= 32) {
+    int pos = w.qn + inc - mine;
+#pragma unroll
+    for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+      for (int e = 0; e < EXP_VEC; ++e) {
+        const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+        if (v[u][e] >= w.thr_f && tok < end) queue[pos++] = cand_key(v[u][e], (uint32_t)tok);
+      }
+    w.qn += total;
+    __syncwarp();
+    if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; }
+  } else {
+    // many elements at or above the threshold (equal logits, or a cold threshold): one
+    // register slot at a time, folding whenever 32 keys are waiting
+#pragma unroll
+    for (int u = 0; u < EXP_UNROLL; ++u) {
+#pragma unroll
+      for (int e = 0; e < EXP_VEC; ++e) {
+        const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+        const bool ok = v[u][e] >= w.thr_f && tok < end;
+        const unsigned mk = __ballot_sync(FULL, ok);
+        if (mk == 0u) continue;
+        if (ok) queue[w.qn + __popc(mk & ((1u << lane) - 1u))] = cand_key(v[u][e], (uint32_t)tok);
+        w.qn += __popc(mk);
+        __syncwarp();
+        if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; }
+      }
+    }
+  }
+}
+
+// The warp's best keys (list and queue) -> the CTA pool.
+__device__ __forceinline__ void pool_from_warp(WarpTopk &w, u64 *queue, u64 *s_pool, int *s_pool_n, int k) {
+  const int lane = threadIdx.x & 31;
+  int cnt_w = w.qn;
+  if (w.folded) {
+    if (w.qn > 0) w.list = warp_merge_desc(w.list, lane < w.qn ? queue[lane] : 0ull, lane);
+    cnt_w = __popc(__ballot_sync(FULL, lane < k && w.list != 0ull));
+  }
+  int pos = 0;
+  if (lane == 0) pos = atomicAdd(s_pool_n, cnt_w);
+  pos = __shfl_sync(FULL, pos, 0);
+  if (lane < cnt_w) s_pool[pos + lane] = w.folded ? w.list : queue[lane];
+}
+
+__device__ __forceinline__ void load_tile(float (&v)[EXP_UNROLL][EXP_VEC], const float *rowp, int base, int end) {
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int u = 0; u < EXP_UNROLL; ++u) {
+    const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+    if (idx + EXP_VEC <= end) {
+      const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
+      v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(EXP_THREADS)
 expand_fused_kernel(FusedArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ u64 s_queue[EXP_WARPS][FX_QCAP];       // per-warp queues of keys above the threshold
-  __shared__ u64 s_pool[EXP_WARPS * 32];            // the chunk's candidates: at most 32 per warp
+  __shared__ u64 s_pool[FX_POOL];                   // the chunk's candidates, all warps
   __shared__ int s_base[MAX_BATCH + 1];
   __shared__ int s_warp[EXP_WARPS];
   __shared__ float s_m[EXP_WARPS], s_s[EXP_WARPS];
+  __shared__ float s_gmax[32];                      // maxima of lane groups (single-tile chunks)
   __shared__ u64 s_anchor;
   __shared__ int s_pool_n, s_last, s_cnt, s_bad;
 
@@ -521,6 +628,8 @@ expand_fused_kernel(FusedArgs a) {
   if (tid == 0) s_pool_n = 0;
   const LayerGeom g = balanced_geom(fr.total, a.V, a.target_items, a.max_splits, a.items_cap);
   const int n_items = fr.total * g.splits;
+  // lanes per group whose maxima bound the k-th largest element of a single-tile chunk
+  const int grp = k <= 8 ? 32 : (k <= 16 ? 16 : 8);
   __syncthreads();
 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -534,70 +643,46 @@ expand_fused_kernel(FusedArgs a) {
     const float *rowp = a.logits + ((int64_t)rl.b * a.rows_per_seq + rsel) * a.row_stride;
     const int start = chunk * g.chunk_len;
     const int end = min(a.V, start + g.chunk_len);
-
-    float m_t = -CUDART_INF_F, s_t = 0.f;
-    u64 list = 0ull;                 // lane p holds the warp's p-th best key so far (once folded)
-    bool folded = false;
-    int qn = 0;                      // keys waiting in this warp's queue (< 32 between tiles)
-    float thr0 = -CUDART_INF_F, thr_f = -CUDART_INF_F;
-    bool first = true;
     u64 *queue = s_queue[warp];
+    float wm, ws;                    // this warp's maximum and sum of exponentials relative to it
 
-
-    for (int base = start; base < end; base += EXP_TILE) {
+    if (end - start <= EXP_TILE) {
+      // ---- the whole chunk in registers ----
       float v[EXP_UNROLL][EXP_VEC];
-#pragma unroll
-      for (int u = 0; u < EXP_UNROLL; ++u) {
-        const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
-        if (idx + EXP_VEC <= end) {
-          const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
-          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-        } else {
-#pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
-        }
-      }
+      load_tile(v, rowp, start, end);
       float bm = -CUDART_INF_F;
 #pragma unroll
       for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
         for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
-
-      if (first) {
-        first = false;
-        // k lane maxima are k distinct elements, so the k-th largest lane maximum is a lower
-        // bound of this warp's k-th largest element: nothing below it needs to be looked at.
-        int rank = 0;
+      float g8 = bm;
 #pragma unroll
-        for (int l = 0; l < 32; ++l) {
-          const float o = __shfl_sync(FULL, bm, l);
-          rank += (o > bm) || (o == bm && l < lane);
-        }
-        const unsigned pick = __ballot_sync(FULL, rank == k - 1);
-        if (pick) thr0 = __shfl_sync(FULL, bm, __ffs(pick) - 1);
-        thr_f = thr0;
-      }
-      // running softmax normaliser of this thread's elements
-      if (bm > m_t) {
-        s_t *= exp2f((m_t - bm) * LOG2E_F);
-        m_t = bm;
-      }
-      if (m_t > -CUDART_INF_F) {
-        float acc = 0.f;
+      for (int o = 1; o < 8; o <<= 1) g8 = fmaxf(g8, __shfl_xor_sync(FULL, g8, o));
+      const float g16 = fmaxf(g8, __shfl_xor_sync(FULL, g8, 8));
+      wm = fmaxf(g16, __shfl_xor_sync(FULL, g16, 16));
+      float acc = 0.f;
+      if (wm > -CUDART_INF_F) {
 #pragma unroll
         for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - m_t) * LOG2E_F);
-        s_t += acc;
+          for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - wm) * LOG2E_F);
       }
-      // top-k: elements that reach the threshold go to the warp's queue
+      ws = acc;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
+      if ((lane & (grp - 1)) == 0) s_gmax[(tid / grp)] = grp == 32 ? wm : (grp == 16 ? g16 : g8);
+      if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
+      __syncthreads();
+      // the smallest group maximum: at least 256/grp >= k elements of the chunk reach it
+      float tau = lane < EXP_THREADS / grp ? s_gmax[lane] : CUDART_INF_F;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) tau = fminf(tau, __shfl_xor_sync(FULL, tau, o));
       int mine = 0;
 #pragma unroll
       for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
         for (int e = 0; e < EXP_VEC; ++e)
-          mine += (v[u][e] >= thr_f && base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
-      if (!__any_sync(FULL, mine > 0)) continue;
+          mine += (v[u][e] >= tau && start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
       int inc = mine;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -605,66 +690,83 @@ expand_fused_kernel(FusedArgs a) {
         if (lane >= o) inc += t;
       }
       const int total = __shfl_sync(FULL, inc, 31);
-      if (total <= 32) {
-        int pos = qn + inc - mine;
+      int pos = 0;
+      if (lane == 0 && total > 0) pos = atomicAdd(&s_pool_n, total);
+      pos = __shfl_sync(FULL, pos, 0) + inc - mine;
+      if (mine > 0 && pos + mine <= FX_POOL) {
 #pragma unroll
         for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
           for (int e = 0; e < EXP_VEC; ++e) {
-            const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-            if (v[u][e] >= thr_f && tok < end) queue[pos++] = cand_key(v[u][e], (uint32_t)tok);
+            const int tok = start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+            if (v[u][e] >= tau && tok < end) s_pool[pos++] = cand_key(v[u][e], (uint32_t)tok);
           }
-        qn += total;
-        __syncwarp();
-        if (qn >= 32) { fold_queue(list, qn, thr_f, queue, thr0, k, lane); folded = true; }
-      } else {
-        // many elements at or above the threshold (equal logits, or a cold threshold): one
-        // register slot at a time, folding whenever 32 keys are waiting
-#pragma unroll
-        for (int u = 0; u < EXP_UNROLL; ++u) {
-#pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) {
-            const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-            const bool ok = v[u][e] >= thr_f && tok < end;
-            const unsigned mk = __ballot_sync(FULL, ok);
-            if (mk == 0u) continue;
-            if (ok) queue[qn + __popc(mk & ((1u << lane) - 1u))] = cand_key(v[u][e], (uint32_t)tok);
-            qn += __popc(mk);
-            __syncwarp();
-            if (qn >= 32) { fold_queue(list, qn, thr_f, queue, thr0, k, lane); folded = true; }
-          }
-        }
       }
+      __syncthreads();
+      if (s_pool_n > FX_POOL) {
+        // too many elements at the bound (equal logits, masked vocabulary, a tiny chunk): take
+        // the per-warp queue route on the same registers
+        __syncthreads();
+        if (tid == 0) s_pool_n = 0;
+        __syncthreads();
+        WarpTopk w;
+        w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
+        w.thr0 = w.thr_f = -CUDART_INF_F;
+        topk_tile(v, bm, start, end, k, queue, w);
+        pool_from_warp(w, queue, s_pool, &s_pool_n, k);
+        __syncthreads();
+      }
+    } else {
+      // ---- a longer chunk, streamed tile by tile ----
+      float m_t = -CUDART_INF_F, s_t = 0.f;
+      WarpTopk w;
+      w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
+      w.thr0 = w.thr_f = -CUDART_INF_F;
+      for (int base = start; base < end; base += EXP_TILE) {
+        float v[EXP_UNROLL][EXP_VEC];
+        load_tile(v, rowp, base, end);
+        float bm = -CUDART_INF_F;
+#pragma unroll
+        for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+          for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
+        // running softmax normaliser of this thread's elements
+        if (bm > m_t) {
+          s_t *= exp2f((m_t - bm) * LOG2E_F);
+          m_t = bm;
+        }
+        if (m_t > -CUDART_INF_F) {
+          float acc = 0.f;
+#pragma unroll
+          for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+            for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - m_t) * LOG2E_F);
+          s_t += acc;
+        }
+        topk_tile(v, bm, base, end, k, queue, w);
+      }
+      pool_from_warp(w, queue, s_pool, &s_pool_n, k);
+      wm = m_t;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(FULL, wm, o));
+      // thread partial rescaled to the warp maximum; a NaN partial (NaN or +inf logit) propagates
+      ws = (m_t > -CUDART_INF_F || s_t != s_t) ? s_t * exp2f((m_t - wm) * LOG2E_F) : 0.f;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
+      if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
+      __syncthreads();
     }
 
-    // ---- this warp's candidates -> the CTA pool; (max, sum) -> shared ----
-    int cnt_w = qn;
-    if (folded) {
-      if (qn > 0) list = warp_merge_desc(list, lane < qn ? queue[lane] : 0ull, lane);
-      cnt_w = __popc(__ballot_sync(FULL, lane < k && list != 0ull));
-    }
-    int pos = 0;
-    if (lane == 0) pos = atomicAdd(&s_pool_n, cnt_w);
-    pos = __shfl_sync(FULL, pos, 0);
-    if (lane < cnt_w) s_pool[pos + lane] = folded ? list : queue[lane];
-    float wm = m_t;
-#pragma unroll
-    for (int o = 16; o; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(FULL, wm, o));
-    // thread partial rescaled to the warp maximum; a NaN partial (NaN or +inf logit) propagates
-    float ws = (m_t > -CUDART_INF_F || s_t != s_t) ? s_t * exp2f((m_t - wm) * LOG2E_F) : 0.f;
-#pragma unroll
-    for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
-    if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
-    __syncthreads();
-
-    // ---- the chunk's k best keys (rank by counting: keys are unique) and its (max, sum) ----
+    // ---- the chunk's k best keys: four lanes count each candidate's betters (keys are unique) ----
     const int nc = s_pool_n;
-    if (tid < nc) {
-      const u64 key = s_pool[tid];
+    for (int c0 = 0; c0 < nc; c0 += EXP_THREADS / 4) {
+      const int ci = c0 + (tid >> 2), q = tid & 3;
+      const u64 key = ci < nc ? s_pool[ci] : 0ull;
       int r = 0;
-#pragma unroll 4
-      for (int o = 0; o < nc; ++o) r += (s_pool[o] > key) ? 1 : 0;
-      if (r < k) a.part_keys[(size_t)item * a.key_stride + r] = key;
+      for (int o = q; o < nc; o += 4) r += (s_pool[o] > key) ? 1 : 0;
+      r += __shfl_xor_sync(FULL, r, 1);
+      r += __shfl_xor_sync(FULL, r, 2);
+      if (q == 0 && ci < nc && r < k) a.part_keys[(size_t)item * a.key_stride + r] = key;
     }
     if (tid >= nc && tid < k) a.part_keys[(size_t)item * a.key_stride + tid] = 0ull;
     if (warp == EXP_WARPS - 1) {
@@ -679,22 +781,22 @@ expand_fused_kernel(FusedArgs a) {
       if (lane == 0) a.part_ms[item] = make_float2(bmx, tot);
     }
 
-    // ---- the last chunk of a sequence runs that sequence's selection ----
-    __threadfence();
+    // ---- the last chunk of a sequence runs that sequence's selection.  The barrier orders
+    // this CTA's writes before thread 0's device-scope release; the last arrival acquires. ----
     __syncthreads();
     if (tid == 0) {
       s_pool_n = 0;
-      const unsigned prev = atomicAdd(&a.seq_count[rl.b], 1u);
+      cuda::atomic_ref<unsigned int, cuda::thread_scope_device> cnt(a.seq_count[rl.b]);
+      const unsigned prev = cnt.fetch_add(1u, cuda::memory_order_acq_rel);
       s_last = (prev == (unsigned)(rl.F * g.splits) - 1u);
-      if (s_last) a.seq_count[rl.b] = 0u;            // ready for the next layer
+      if (s_last) cnt.store(0u, cuda::memory_order_relaxed);      // ready for the next layer
     }
     __syncthreads();
     if (!s_last) continue;
-    __threadfence();
     TailSmem sm;
     const int rows_max = a.N - 1;
     unsigned char *p = smem_raw;
-    sm.stage = reinterpret_cast<u64 *>(p);            p += sizeof(u64) * EXP_WARPS * FX_STAGE;
+    sm.stage = reinterpret_cast<u64 *>(p);            p += sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV);
     sm.row_keys = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * k;
     sm.score = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max * k;
     sm.row_t = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max;
@@ -710,14 +812,14 @@ expand_fused_kernel(FusedArgs a) {
 
 size_t fused_smem_bytes(const talon_ctx *c) {
   const size_t rows = c->p.budget - 1, k = c->k_cap, W = c->W;
-  return sizeof(u64) * EXP_WARPS * FX_STAGE + rows * k * (8 + 8 + 1) + rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
+  return sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV) + rows * k * (8 + 8 + 1) + rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
 }
 
 }  // namespace
 
 int fused_max_splits(int key_stride) {
-  int s = FX_STAGE / (2 * key_stride);          // half of a warp's staging area stays free for survivors
-  return s > FX_MAX_SPLITS ? FX_MAX_SPLITS : (s < 1 ? 1 : s);
+  (void)key_stride;
+  return FX_MAX_SPLITS;
 }
 
 talon_status expand_fused_setup(talon_ctx *c) {

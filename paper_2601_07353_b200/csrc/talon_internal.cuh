@@ -27,8 +27,9 @@ constexpr int MAX_BATCH = 1024;
 constexpr int SEL_THREADS = 512;
 // fused expansion kernel (k <= 32)
 constexpr int FX_QCAP = 64;                // keys a warp's queue can hold
-constexpr int FX_STAGE = 512;              // keys a warp stages while merging one row's chunk lists
-constexpr int FX_MAX_SPLITS = 64;          // chunks per row, at most
+constexpr int FX_SURV = 64;                // keys of a row that may pass the merge bound before the slow path
+constexpr int FX_MAX_SPLITS = 32;          // chunks per row, at most (one lane per chunk in the merge)
+constexpr int FX_POOL = 256;               // candidates a CTA can pool for one chunk
 
 // Order-preserving map fp32 -> u32 (larger float <=> larger integer; -inf > 0).
 __host__ __device__ inline uint32_t f32_ord(float f) {
