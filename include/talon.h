@@ -211,6 +211,28 @@ talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const
                         int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
                         void *stream);
 
+/* The paper has no counterpart for this call: it exists for callers that cannot allocate.
+ * talon_accept needs a context, and talon_create calls cudaMalloc.  Code that runs inside a
+ * fixed memory pool, or in a part of a serving loop where allocating is not allowed (it
+ * synchronises the device and may fail when memory is tight), can use this call instead for the
+ * first half of the greedy verification: t_i = argmax of target-logit row i, lowest id among
+ * equal maxima, -1 for a row that holds only NaN.  It needs no context and calls no cudaMalloc,
+ * cudaFree or any other allocating routine; its scratch (one 8-byte key per row) is a fixed
+ * array inside the library image, TALON_NOALLOC_MAX_ROWS * 8 bytes on every GPU that loads the
+ * library, held until the process exits.
+ *  target_logits device fp32, row i at target_logits + i * row_stride; 16-byte aligned
+ *  row_stride    elements between rows, a multiple of 4 and >= vocab
+ *  n_rows        0 .. TALON_NOALLOC_MAX_ROWS; more returns TALON_ERR_CAPACITY, nothing enqueued
+ *  target_tok    device [n_rows]
+ * Runs on the current device; enqueues three kernels on `stream` and returns.  The first call on
+ * a device looks up the array's device address (cudaGetSymbolAddress) and the SM count; make
+ * that first call outside any stream capture.  Every call clears the rows it uses first, since
+ * the array keeps the previous call's keys.  All calls share the one array: two calls that can
+ * overlap on the GPU (different streams without an ordering between them) race. */
+#define TALON_NOALLOC_MAX_ROWS 8192
+talon_status talon_target_argmax_noalloc(const float *target_logits, int64_t row_stride, int32_t vocab,
+                                         int32_t n_rows, int32_t *target_tok, void *stream);
+
 /* Number of kernels the library has launched through this context since creation. */
 int64_t talon_launch_count(const talon_ctx *ctx);
 

@@ -55,19 +55,21 @@ _lib.talon_timing_enable.argtypes = [_vp, _i32, C.c_uint32]
 _lib.talon_timing_read.argtypes = [_vp, _vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.talon_kernel_name.argtypes = [_i32]
 _lib.talon_kernel_name.restype = C.c_char_p
+_lib.talon_target_argmax_noalloc.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp]
 _lib.talon_launch_count.argtypes = [_vp]
 _lib.talon_launch_count.restype = C.c_int64
 _lib.talon_status_string.argtypes = [C.c_int]
 _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
-           "talon_step", "talon_timing_enable", "talon_timing_read"):
+           "talon_step", "talon_timing_enable", "talon_timing_read", "talon_target_argmax_noalloc"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
             "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
             "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_kernel_name",
-            "talon_launch_count", "talon_status_string"]
+            "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc"]
+NOALLOC_MAX_ROWS = 8192
 N_KERNELS = 8
 KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
 
@@ -89,6 +91,18 @@ def _ptr(t: Optional[torch.Tensor]):
 
 def _stream(device) -> C.c_void_p:
     return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def target_argmax_noalloc(target_logits: torch.Tensor, target_tok: torch.Tensor) -> None:
+    """``talon_target_argmax_noalloc``: greedy target token of every row of ``target_logits``
+    ([rows, V] fp32 on the current CUDA device) into ``target_tok`` ([rows] int32), with no context
+    and no allocation in the library: for callers that are not allowed to call cudaMalloc.  At most
+    ``NOALLOC_MAX_ROWS`` rows; the library's single scratch array is shared by all calls, so calls
+    must not overlap on the GPU."""
+    rows = target_logits.numel() // target_logits.shape[-1]
+    _check(_lib.talon_target_argmax_noalloc(_ptr(target_logits), target_logits.stride(-2), target_logits.shape[-1],
+                                            rows, _ptr(target_tok), _stream(target_logits.device)),
+           "talon_target_argmax_noalloc")
 
 
 @dataclass
