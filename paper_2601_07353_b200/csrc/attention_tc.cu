@@ -78,8 +78,9 @@ __device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ inline bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  // the hint lets the hardware park the thread until the phase completes (or ~20 us pass)
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return ok != 0;
 }
 // Waits for the phase with the given parity; gives up after TC_WAIT_CYCLES or when another

@@ -46,6 +46,42 @@ struct FusedArgs {
   int *status;
 };
 
+// 2^x on the special-function unit (relative error about 2^-22, results below 2^-126 flush to 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- bulk-copy ring: a longer chunk is brought in by the TMA engine, FX_RING tiles ahead ----
+__device__ inline uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ inline void ring_bar_init(uint32_t bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+}
+// Arms `bar` for `bytes` and starts the copy global -> shared (both 16-byte aligned, bytes a
+// multiple of 16).  No multicast.
+__device__ inline void ring_issue(uint32_t dst, const float *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Waits for the phase of `bar` with the given parity, for about two seconds at most.
+__device__ inline bool ring_wait(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i) {
+      uint32_t ok;
+      // the hint lets the hardware park the thread until the phase completes (or ~20 us pass)
+      asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}"
+                   : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+      if (ok) return true;
+    }
+    if (clock64() - t0 > 4000000000ll) return false;
+  }
+}
+
 __device__ inline u64 shfl_u64(u64 v, int src) { return __shfl_sync(FULL, v, src); }
 __device__ inline u64 shfl_xor_u64(u64 v, int m) { return __shfl_xor_sync(FULL, v, m); }
 __device__ inline u64 umax64(u64 a, u64 b) { return a > b ? a : b; }
@@ -83,16 +119,33 @@ __device__ inline u64 warp_merge_desc(u64 list, u64 q, int lane) {
   return x;
 }
 
-// Folds the first 32 queued keys into the warp's list, moves the rest of the queue to its front
-// and raises the threshold to the list's k-th key.
+// Folds the first 32 queued keys into the warp's list, moves the rest of the queue (up to
+// FX_QCAP - 32 keys) to its front and raises the threshold to the list's k-th key.
 __device__ __forceinline__ void fold_queue(u64 &list, int &qn, float &thr_f, u64 *queue, float thr0, int k,
                                            int lane) {
   list = warp_merge_desc(list, queue[lane], lane);
-  const u64 rest = queue[32 + lane];
+  const int rem = qn - 32;
+  const u64 r0 = queue[32 + lane], r1 = queue[64 + lane], r2 = queue[96 + lane];
   __syncwarp();
-  qn -= 32;
-  if (lane < qn) queue[lane] = rest;
+  if (lane < rem) queue[lane] = r0;
+  if (32 + lane < rem) queue[32 + lane] = r1;
+  if (64 + lane < rem) queue[64 + lane] = r2;
   __syncwarp();
+  qn = rem;
+  const u64 kth = shfl_u64(list, k - 1);
+  if (kth) thr_f = fmaxf(thr0, key_logit(kth));
+}
+
+// Makes a warp's threshold known to the other warps of the CTA (monotone: a maximum).
+__device__ __forceinline__ void publish_thr(unsigned *thr_cta, float thr_f, int lane) {
+  if (lane == 0 && thr_f > -CUDART_INF_F) atomicMax(thr_cta, f32_ord(thr_f));
+}
+
+// Folds a queue of fewer than 32 keys into the list (queue left empty).
+__device__ __forceinline__ void flush_queue(u64 &list, int &qn, float &thr_f, const u64 *queue, float thr0, int k,
+                                            int lane) {
+  list = warp_merge_desc(list, lane < qn ? queue[lane] : 0ull, lane);
+  qn = 0;
   const u64 kth = shfl_u64(list, k - 1);
   if (kth) thr_f = fmaxf(thr0, key_logit(kth));
 }
@@ -274,7 +327,55 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
   // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys.
   // One warp per row, one lane per chunk (S <= 32). ----
   const int stage_words = 32 * k + FX_SURV;
-  for (int j = warp; j < F; j += EXP_WARPS) {
+  // Many rows means few chunks per row (their product is bounded by the grid): then all rows
+  // are merged at once, one thread per key, instead of a row at a time per warp.
+  const bool flat = S > 1 && S <= 8 && F > EXP_WARPS && F * S * k <= EXP_WARPS * stage_words;
+  if (flat) {
+    const size_t item0 = (size_t)row0 * S;
+    u64 *st = sm.stage;                           // st[(j * S + c) * k + i]
+    const int nkeys = F * S * k;
+    for (int idx = tid; idx < nkeys; idx += EXP_THREADS) {
+      const int jc = idx / k, i = idx - jc * k;
+      st[idx] = __ldcg(a.part_keys + (item0 + jc) * ks + i);
+    }
+    for (int idx = tid; idx < F * k; idx += EXP_THREADS) sm.row_keys[idx] = 0ull;
+    for (int j = tid; j < F; j += EXP_THREADS) {
+      sm.row_ps[j] = a.t.score[nb + lo + j];
+      for (int w = 0; w < a.W; ++w) sm.row_mask[j * a.W + w] = a.t.mask[(nb + lo + j) * a.W + w];
+      float mx = -CUDART_INF_F;
+      for (int c = 0; c < S; ++c) mx = fmaxf(mx, __ldcg(a.part_ms + item0 + (size_t)j * S + c).x);
+      double t = 0.0;
+      for (int c = 0; c < S; ++c) {
+        const float2 ms = __ldcg(a.part_ms + item0 + (size_t)j * S + c);
+        if (ms.y != ms.y) t += (double)ms.y;                              // NaN or +inf logit in the chunk
+        else if (ms.x > -CUDART_INF_F) t += (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
+      }
+      sm.row_m[j] = mx;
+      sm.row_t[j] = t;
+    }
+    __syncthreads();
+    // a key's rank in its row: its place in its own list plus, for every other chunk of the
+    // row, how many of that chunk's keys beat it (keys are unique; lists are descending)
+    for (int idx = tid; idx < nkeys; idx += EXP_THREADS) {
+      const u64 key = st[idx];
+      if (key == 0ull) continue;
+      const int jc = idx / k, i = idx - jc * k;
+      const int j = jc / S, c = jc - j * S;
+      int rank = i;
+      for (int o = 0; o < S; ++o) {
+        if (o == c) continue;
+        const u64 *lst = st + (size_t)(j * S + o) * k;
+        int l = 0, h = k;
+        while (l < h) {
+          const int mid = (l + h) >> 1;
+          if (lst[mid] > key) l = mid + 1; else h = mid;
+        }
+        rank += l;
+      }
+      if (rank < k) sm.row_keys[(size_t)j * k + rank] = key;
+    }
+  }
+  for (int j = flat ? F : warp; j < F; j += EXP_WARPS) {
     const size_t item0 = (size_t)(row0 + j) * S;
     u64 *st = sm.stage + warp * stage_words;       // st[i * 32 + c] = i-th best key of chunk c
     u64 *sv = st + 32 * k;                         // keys that reach the bound
@@ -490,8 +591,9 @@ struct WarpTopk {
 // One tile (16 elements per thread, already in registers) through the warp's threshold queue.
 // bm is the thread's maximum over the tile.
 __device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC], float bm, int base, int end, int k,
-                                          u64 *queue, WarpTopk &w) {
+                                          u64 *queue, int *qcnt, unsigned *thr_cta, WarpTopk &w) {
   const int tid = threadIdx.x, lane = tid & 31;
+  const bool was_first = w.first;
   if (w.first) {
     w.first = false;
     // k lane maxima are k distinct elements, so the k-th largest lane maximum is a lower
@@ -505,6 +607,35 @@ __device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC],
     const unsigned pick = __ballot_sync(FULL, rank == k - 1);
     if (pick) w.thr0 = __shfl_sync(FULL, bm, __ffs(pick) - 1);
     w.thr_f = w.thr0;
+  }
+  // A thread holds something at or above the threshold iff its maximum over the tile is: one
+  // compare per tile.  The threshold is shared by the CTA's warps: whenever a warp sorts its
+  // keys, its k-th best key is a lower bound of the chunk's k-th largest element for everybody.
+  {
+    const unsigned shared_thr = *thr_cta;
+    if (shared_thr) w.thr_f = fmaxf(w.thr_f, f32_unord(shared_thr));
+  }
+  const bool hit = bm >= w.thr_f;
+  const unsigned hm = __ballot_sync(FULL, hit);
+  if (hm == 0u) return;
+  if (__popc(hm) <= 6) {
+    // a few lanes hold everything that reaches the threshold: only they look at their elements
+    // (at most 6 x 16 new keys; fewer than 32 were waiting)
+    if (lane == 0) *qcnt = w.qn;
+    __syncwarp();
+    if (hit) {
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+        for (int e = 0; e < EXP_VEC; ++e) {
+          const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+          if (v[u][e] >= w.thr_f && tok < end) queue[atomicAdd(qcnt, 1)] = cand_key(v[u][e], (uint32_t)tok);
+        }
+    }
+    __syncwarp();
+    w.qn = *qcnt;
+    while (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
+    return;
   }
   int mine = 0;
 #pragma unroll
@@ -531,7 +662,14 @@ __device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC],
       }
     w.qn += total;
     __syncwarp();
-    if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; }
+    if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
+    else if (was_first && w.qn >= k) {
+      // the first tile's bound is loose: sort what it let through so that the k-th best key of
+      // this tile becomes the threshold for the next ones
+      flush_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane);
+      w.folded = true;
+      publish_thr(thr_cta, w.thr_f, lane);
+    }
   } else {
     // many elements at or above the threshold (equal logits, or a cold threshold): one
     // register slot at a time, folding whenever 32 keys are waiting
@@ -546,7 +684,7 @@ __device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC],
         if (ok) queue[w.qn + __popc(mk & ((1u << lane) - 1u))] = cand_key(v[u][e], (uint32_t)tok);
         w.qn += __popc(mk);
         __syncwarp();
-        if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; }
+        if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
       }
     }
   }
@@ -581,14 +719,17 @@ __device__ __forceinline__ void load_tile(float (&v)[EXP_UNROLL][EXP_VEC], const
   }
 }
 
-__global__ void __launch_bounds__(EXP_THREADS)
+__global__ void __launch_bounds__(EXP_THREADS, 3)
 expand_fused_kernel(FusedArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ u64 s_queue[EXP_WARPS][FX_QCAP];       // per-warp queues of keys above the threshold
   __shared__ u64 s_pool[FX_POOL];                   // the chunk's candidates, all warps
   __shared__ int s_base[MAX_BATCH + 1];
   __shared__ int s_warp[EXP_WARPS];
   __shared__ float s_m[EXP_WARPS], s_s[EXP_WARPS];
+  __shared__ __align__(8) unsigned long long s_ring_bar[FX_RING];   // "tile landed" barriers
+  __shared__ unsigned s_thr_cta;                    // ordered bits of the CTA-wide threshold (0: none yet)
+  __shared__ int s_qn[EXP_WARPS];                   // queue fill, when lanes append on their own
   __shared__ float s_gmax[32];                      // maxima of lane groups (single-tile chunks)
   __shared__ u64 s_anchor;
   __shared__ int s_pool_n, s_last, s_cnt, s_bad;
@@ -625,7 +766,13 @@ expand_fused_kernel(FusedArgs a) {
       for (int b = tid; b < a.B; b += EXP_THREADS)
         if (s_base[b + 1] == s_base[b]) a.t.layer_off[b * a.lo_stride + a.d + 2] = a.t.n_nodes[b];
   }
-  if (tid == 0) s_pool_n = 0;
+  if (tid == 0) {
+    s_pool_n = 0;
+    s_thr_cta = 0u;
+    for (int i = 0; i < FX_RING; ++i) ring_bar_init(smem_addr(&s_ring_bar[i]));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  unsigned ring_tiles = 0;         // tiles this CTA has taken from the ring so far (all threads agree)
   const LayerGeom g = balanced_geom(fr.total, a.V, a.target_items, a.max_splits, a.items_cap);
   const int n_items = fr.total * g.splits;
   // lanes per group whose maxima bound the k-th largest element of a single-tile chunk
@@ -665,7 +812,7 @@ expand_fused_kernel(FusedArgs a) {
 #pragma unroll
         for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - wm) * LOG2E_F);
+          for (int e = 0; e < EXP_VEC; ++e) acc += fast_exp2(fmaf(v[u][e], LOG2E_F, -wm * LOG2E_F));
       }
       ws = acc;
 #pragma unroll
@@ -712,7 +859,7 @@ expand_fused_kernel(FusedArgs a) {
         WarpTopk w;
         w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
         w.thr0 = w.thr_f = -CUDART_INF_F;
-        topk_tile(v, bm, start, end, k, queue, w);
+        topk_tile(v, bm, start, end, k, queue, &s_qn[warp], &s_thr_cta, w);
         pool_from_warp(w, queue, s_pool, &s_pool_n, k);
         __syncthreads();
       }
@@ -722,9 +869,46 @@ expand_fused_kernel(FusedArgs a) {
       WarpTopk w;
       w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
       w.thr0 = w.thr_f = -CUDART_INF_F;
-      for (int base = start; base < end; base += EXP_TILE) {
+      const int nt = (end - start + EXP_TILE - 1) / EXP_TILE;
+      float *ring = reinterpret_cast<float *>(smem_raw);        // FX_RING tiles; the selection phase reuses it
+      auto issue = [&](int t, unsigned slot_index) {
+        const int base = start + t * EXP_TILE;
+        const int n = min(EXP_TILE, end - base);
+        const unsigned st = slot_index % FX_RING;
+        // whole 16-byte units: the last one may reach into the row's stride padding
+        ring_issue(smem_addr(ring + st * EXP_TILE), rowp + base, (uint32_t)(((n * 4) + 15) & ~15),
+                   smem_addr(&s_ring_bar[st]));
+      };
+      if (tid == 0)
+        for (int t = 0; t < nt && t < FX_RING; ++t) issue(t, ring_tiles + t);
+      for (int t = 0; t < nt; ++t) {
+        const int base = start + t * EXP_TILE;
+        const unsigned st = ring_tiles % FX_RING;
+        const bool landed = ring_wait(smem_addr(&s_ring_bar[st]), (ring_tiles / FX_RING) & 1u);
         float v[EXP_UNROLL][EXP_VEC];
-        load_tile(v, rowp, base, end);
+#pragma unroll
+        for (int u = 0; u < EXP_UNROLL; ++u) {
+          const int off = u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+          const float4 x = *reinterpret_cast<const float4 *>(ring + st * EXP_TILE + off);
+          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+        }
+        if (base + EXP_TILE > end) {          // the chunk's last, partial tile: nothing past `end` counts
+#pragma unroll
+          for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+            for (int e = 0; e < EXP_VEC; ++e)
+              if (base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e >= end) v[u][e] = -CUDART_INF_F;
+        }
+        // every thread has its copy of the tile: the slot can take the tile FX_RING ahead
+        if (!__syncthreads_and(landed)) {
+          if (tid == 0) atomicOr(a.status, STATUS_TIMEOUT);
+          return;
+        }
+        if (tid == 0 && t + FX_RING < nt) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          issue(t + FX_RING, ring_tiles + FX_RING);
+        }
+        ++ring_tiles;
         float bm = -CUDART_INF_F;
 #pragma unroll
         for (int u = 0; u < EXP_UNROLL; ++u)
@@ -732,18 +916,20 @@ expand_fused_kernel(FusedArgs a) {
           for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
         // running softmax normaliser of this thread's elements
         if (bm > m_t) {
-          s_t *= exp2f((m_t - bm) * LOG2E_F);
+          s_t *= fast_exp2((m_t - bm) * LOG2E_F);
           m_t = bm;
         }
         if (m_t > -CUDART_INF_F) {
+          // exp(v - m) = 2^(v * log2e - m * log2e); an infinite m (a +inf logit) must give NaN
+          const float c = -m_t * LOG2E_F;
           float acc = 0.f;
 #pragma unroll
           for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
-            for (int e = 0; e < EXP_VEC; ++e) acc += exp2f((v[u][e] - m_t) * LOG2E_F);
+            for (int e = 0; e < EXP_VEC; ++e) acc += fast_exp2(fmaf(v[u][e], LOG2E_F, c));
           s_t += acc;
         }
-        topk_tile(v, bm, base, end, k, queue, w);
+        topk_tile(v, bm, base, end, k, queue, &s_qn[warp], &s_thr_cta, w);
       }
       pool_from_warp(w, queue, s_pool, &s_pool_n, k);
       wm = m_t;
@@ -786,6 +972,7 @@ expand_fused_kernel(FusedArgs a) {
     __syncthreads();
     if (tid == 0) {
       s_pool_n = 0;
+      s_thr_cta = 0u;
       cuda::atomic_ref<unsigned int, cuda::thread_scope_device> cnt(a.seq_count[rl.b]);
       const unsigned prev = cnt.fetch_add(1u, cuda::memory_order_acq_rel);
       s_last = (prev == (unsigned)(rl.F * g.splits) - 1u);
@@ -807,12 +994,16 @@ expand_fused_kernel(FusedArgs a) {
     sm.row_off = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
     sm.state = p;
     select_tail(a, sm, rl.b, rl.row0, rl.F, g.splits, &s_anchor, &s_cnt, &s_bad);
+    __syncthreads();     // the next chunk's bulk copies land in the memory the selection phase just used
   }
 }
 
 size_t fused_smem_bytes(const talon_ctx *c) {
   const size_t rows = c->p.budget - 1, k = c->k_cap, W = c->W;
-  return sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV) + rows * k * (8 + 8 + 1) + rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
+  const size_t tail = sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV) + rows * k * (8 + 8 + 1) +
+                      rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
+  const size_t ring = sizeof(float) * FX_RING * EXP_TILE;       // the two phases share the space
+  return tail > ring ? tail : ring;
 }
 
 }  // namespace

@@ -26,9 +26,10 @@ constexpr int MAX_BUDGET = 128;
 constexpr int MAX_BATCH = 1024;
 constexpr int SEL_THREADS = 512;
 // fused expansion kernel (k <= 32)
-constexpr int FX_QCAP = 64;                // keys a warp's queue can hold
+constexpr int FX_QCAP = 128;               // keys a warp's queue can hold
 constexpr int FX_SURV = 64;                // keys of a row that may pass the merge bound before the slow path
 constexpr int FX_MAX_SPLITS = 32;          // chunks per row, at most (one lane per chunk in the merge)
+constexpr int FX_RING = 3;                 // 16 KB tiles in flight per CTA on the streaming path
 constexpr int FX_POOL = 256;               // candidates a CTA can pool for one chunk
 
 // Order-preserving map fp32 -> u32 (larger float <=> larger integer; -inf > 0).
