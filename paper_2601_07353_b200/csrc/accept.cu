@@ -27,6 +27,7 @@ struct ArgmaxArgs {
 __global__ void __launch_bounds__(EXP_THREADS)
 target_argmax_kernel(ArgmaxArgs a) {
   __shared__ unsigned long long s_key[EXP_WARPS];
+  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_items = a.B * a.N * a.splits;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
@@ -95,6 +96,7 @@ struct WalkArgs {
 
 // one warp per sequence
 __global__ void accept_walk_kernel(WalkArgs a) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (b >= a.B) return;
@@ -146,7 +148,7 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   if (items < grid) grid = (int)items;
   {
     LaunchTimer lt(c, TALON_K_ARGMAX, st);
-    target_argmax_kernel<<<grid, EXP_THREADS, 0, st>>>(aa);
+    launch_kernel(c, target_argmax_kernel, dim3(grid), dim3(EXP_THREADS), 0, st, aa);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
 
@@ -158,7 +160,7 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   const int warps_per_block = 4;
   {
     LaunchTimer lt(c, TALON_K_WALK, st);
-    accept_walk_kernel<<<(c->B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(wa);
+    launch_kernel(c, accept_walk_kernel, dim3((c->B + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, st, wa);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 2;

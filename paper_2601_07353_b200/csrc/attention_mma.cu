@@ -81,6 +81,7 @@ __device__ inline void load_kv_tile(unsigned char *dst, const __nv_bfloat16 *src
 
 __global__ void __launch_bounds__(AT_THREADS, 1)
 tree_attention_mma_kernel(AttnArgs a) {
+  pdl_enter();
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_q = smem;
   unsigned char *s_kv = smem + AT_BM * AT_D * 2;     // stage s: K at s*2*TILE, V at (s*2+1)*TILE
@@ -291,6 +292,7 @@ tree_attention_mma_kernel(AttnArgs a) {
 
 // merge the split-KV partials: one warp per packed query row
 __global__ void attention_combine_kernel(AttnArgs a) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int mpad = a.m_blocks * AT_BM;
   const int rows_total = a.g * a.N;
@@ -377,7 +379,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
       const int64_t rows = (int64_t)c->B * a.Hkv * a.g * a.N;
       const int wpb = 8;
       LaunchTimer lt(c, TALON_K_COMBINE, st);
-      attention_combine_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(a);
+      launch_kernel(c, attention_combine_kernel, dim3((unsigned)((rows + wpb - 1) / wpb)), dim3(wpb * 32), 0, st, a);
       if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
       c->launches += 1;
     }
@@ -399,7 +401,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
   dim3 grid(a.m_blocks, splits, c->B * a.Hkv);
   {
     LaunchTimer lt(c, TALON_K_ATTENTION, st);
-    tree_attention_mma_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(a);
+    launch_kernel(c, tree_attention_mma_kernel, grid, dim3(AT_THREADS), AT_SMEM, st, a);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;
@@ -407,7 +409,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
     const int64_t rows = (int64_t)c->B * a.Hkv * a.g * a.N;
     const int wpb = 8;
     LaunchTimer lt(c, TALON_K_COMBINE, st);
-    attention_combine_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(a);
+    launch_kernel(c, attention_combine_kernel, dim3((unsigned)((rows + wpb - 1) / wpb)), dim3(wpb * 32), 0, st, a);
     if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
     c->launches += 1;
   }

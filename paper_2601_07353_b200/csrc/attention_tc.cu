@@ -182,6 +182,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
+  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int mpair = blockIdx.x, split = blockIdx.y;
   const int bh = blockIdx.z, b = bh / a.Hkv, kvh = bh - b * a.Hkv;
@@ -596,7 +597,7 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
   dim3 grid((m_blocks + 1) / 2, splits, B * Hkv);
   {
     LaunchTimer lt(c, TALON_K_ATTENTION, st);
-    tree_attention_tc_kernel<<<grid, TC_THREADS, TC_SMEM, st>>>(mq, mkp, mvp, mkt, mvt, a);
+    launch_kernel(c, tree_attention_tc_kernel, grid, dim3(TC_THREADS), TC_SMEM, st, mq, mkp, mvp, mkt, mvt, a);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;

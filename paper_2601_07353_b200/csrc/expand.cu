@@ -183,6 +183,7 @@ expand_rows_kernel(ExpandArgs a) {
   __shared__ float s_bm;
   __shared__ int s_last;
 
+  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   frontier_scan<EXP_THREADS>(a.n_nodes, a.layer_off, a.lo_stride, a.B, a.N, a.d, s_base, s_warp);
   const LayerGeom g = make_geom(s_base[a.B], a.V, a.target_items);
@@ -410,6 +411,7 @@ select_layer_kernel(SelectArgs a) {
   __shared__ int s_cnt, s_need, s_bin, s_done, s_bad;
   __shared__ int s_rowcnt[MAX_BUDGET], s_rowoff[MAX_BUDGET];
 
+  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x;
   frontier_scan<SEL_THREADS>(a.t.n_nodes, a.t.layer_off, a.lo_stride, a.B, a.N, a.d, s_base, s_warp);
@@ -585,6 +587,7 @@ select_layer_kernel(SelectArgs a) {
 __global__ void reset_kernel(talon_tree t, const int32_t *root_tok, const int32_t *prefix_len,
                              int32_t *prefix_copy, int B, int N, int W, int lo_stride, int *status,
                              unsigned int *row_count, int rows_cap, unsigned int *seq_count) {
+  pdl_enter();
   const int gid = blockIdx.x * blockDim.x + threadIdx.x;
   const int stride = gridDim.x * blockDim.x;
   if (gid == 0) *status = 0;
@@ -606,6 +609,7 @@ __global__ void reset_kernel(talon_tree t, const int32_t *root_tok, const int32_
 
 __global__ void build_tree_kernel(talon_tree t, const int32_t *prefix_len, uint8_t *dense, int B, int N,
                                   int W, int lo_stride, int layers_run) {
+  pdl_enter();
   const int b = blockIdx.x;
   const int n = t.n_nodes[b];
   const size_t nb = (size_t)b * N;
@@ -671,8 +675,8 @@ talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root
   if (blocks > 64) blocks = 64;
   if (blocks < 1) blocks = 1;
   LaunchTimer lt(c, TALON_K_RESET, st);
-  reset_kernel<<<blocks, threads, 0, st>>>(*t, root_tok, prefix_len, c->d_prefix_len, B, c->p.budget, c->W,
-                                           c->p.max_depth + 2, c->d_status, c->d_row_count, c->rows_cap, c->d_seq_count);
+  launch_kernel(c, reset_kernel, dim3(blocks), dim3(threads), 0, st, *t, root_tok, prefix_len, c->d_prefix_len, B,
+                c->p.budget, c->W, c->p.max_depth + 2, c->d_status, c->d_row_count, c->rows_cap, c->d_seq_count);
   c->launches += 1;
   return cudaGetLastError() == cudaSuccess ? TALON_OK : TALON_ERR_CUDA;
 }
@@ -699,9 +703,9 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
   {
     LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
     switch (c->k_slots) {
-      case 1: expand_rows_kernel<1><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
-      case 2: expand_rows_kernel<2><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
-      default: expand_rows_kernel<4><<<grid, EXP_THREADS, lists_bytes, st>>>(ea); break;
+      case 1: launch_kernel(c, expand_rows_kernel<1>, dim3(grid), dim3(EXP_THREADS), lists_bytes, st, ea); break;
+      case 2: launch_kernel(c, expand_rows_kernel<2>, dim3(grid), dim3(EXP_THREADS), lists_bytes, st, ea); break;
+      default: launch_kernel(c, expand_rows_kernel<4>, dim3(grid), dim3(EXP_THREADS), lists_bytes, st, ea); break;
     }
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
@@ -715,7 +719,7 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
   sa.pool_cap = pool_capacity(c);
   {
     LaunchTimer lt(c, TALON_K_SELECT, st);
-    select_layer_kernel<<<c->B, SEL_THREADS, select_smem_bytes(sa.pool_cap), st>>>(sa);
+    launch_kernel(c, select_layer_kernel, dim3(c->B), dim3(SEL_THREADS), select_smem_bytes(sa.pool_cap), st, sa);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 2;
@@ -724,8 +728,8 @@ talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logit
 
 talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cudaStream_t st) {
   LaunchTimer lt(c, TALON_K_BUILD, st);
-  build_tree_kernel<<<c->B, 128, 0, st>>>(*t, c->d_prefix_len, dense, c->B, c->p.budget, c->W,
-                                          c->p.max_depth + 2, c->layers_run);
+  launch_kernel(c, build_tree_kernel, dim3(c->B), dim3(128), 0, st, *t, c->d_prefix_len, dense, c->B, c->p.budget,
+                c->W, c->p.max_depth + 2, c->layers_run);
   c->launches += 1;
   return cudaGetLastError() == cudaSuccess ? TALON_OK : TALON_ERR_CUDA;
 }

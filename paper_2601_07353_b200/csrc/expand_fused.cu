@@ -734,6 +734,7 @@ expand_fused_kernel(FusedArgs a) {
   __shared__ u64 s_anchor;
   __shared__ int s_pool_n, s_last, s_cnt, s_bad;
 
+  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = a.k;
 
@@ -1045,7 +1046,7 @@ talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float 
   a.part_keys = c->d_part_keys; a.part_ms = c->d_part_ms; a.seq_count = c->d_seq_count; a.status = c->d_status;
   {
     LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
-    expand_fused_kernel<<<grid, EXP_THREADS, fused_smem_bytes(c), st>>>(a);
+    launch_kernel(c, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c), st, a);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;

@@ -108,6 +108,7 @@ struct talon_ctx {
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int pdl;                           // 1: kernels are launched with programmatic stream serialization
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
   int32_t *d_target_tok;             // [batch_max * N]
@@ -124,6 +125,32 @@ struct talon_ctx {
 };
 
 namespace talon {
+
+// Programmatic dependent launch.  Every kernel of the library starts with pdl_enter(): it lets
+// the next kernel of the stream be scheduled at once and then waits until the previous kernel
+// has completed and its memory is visible, so only launch latency overlaps, never data.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// Launches `kernel` so that it may be scheduled while its predecessor in the stream drains
+// (the kernel itself waits in pdl_enter()); a plain launch when ctx->pdl is off.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = c->pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Brackets one kernel launch with a pair of CUDA events on the launching stream when timing
 // is on; does nothing otherwise.  Pairs beyond the capacity are silently not timed.
