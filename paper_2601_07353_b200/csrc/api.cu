@@ -113,6 +113,9 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     // Programmatic dependent launch is off unless TALON_PDL=1: measured on B200 it gains about 2 %
     // at batch 1 and loses about 10 % at batch 16, where the early-scheduled CTAs of the next
     // kernel take SM slots from the running one.
+    const char *mt = std::getenv("TALON_ATTN_MIN_TILES");
+    c->attn_min_tiles = mt ? std::atoi(mt) : 4;
+    if (c->attn_min_tiles < 1) c->attn_min_tiles = 1;
     const char *e = std::getenv("TALON_PDL");
     c->pdl = (e && e[0] == '1') ? 1 : 0;
   }

@@ -366,7 +366,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
     int sp = 1;
     if (ctas < c->sm_count) {
       sp = c->sm_count / ctas;
-      const int by_tiles = (tiles + TC_MIN_TILES_PER_CTA - 1) / TC_MIN_TILES_PER_CTA;
+      const int by_tiles = (tiles + c->attn_min_tiles - 1) / c->attn_min_tiles;
       if (sp > by_tiles) sp = by_tiles;
       if (sp < 1) sp = 1;
     }

@@ -371,22 +371,29 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       else if (kvalid < 128) see1 &= kvalid == 64 ? 0ull : (~0ull >> (128 - kvalid));
       if (tree_tile && (tg - nP) > 0) { see0 = 0ull; see1 = 0ull; }     // N <= 128: there is one tree tile
 
-      // ---- pass 1: row maximum ----
-      float mx = -CUDART_INF_F;
+      // ---- the row of S: one read from tensor memory, held in registers ----
+      uint32_t r[4][32];
+      tc_ld32(t_S + 0, r[0]);
+      tc_ld32(t_S + 32, r[1]);
+      tc_ld32(t_S + 64, r[2]);
+      tc_ld32(t_S + 96, r[3]);
+      tc_wait_ld();
+      if (masked) {
 #pragma unroll
-      for (int c0 = 0; c0 < TC_BN; c0 += 32) {
-        uint32_t r[32];
-        tc_ld32(t_S + c0, r);
-        tc_wait_ld();
-        if (masked) {
-          const uint32_t bits = (uint32_t)((c0 < 64 ? see0 : see1) >> (c0 & 63));
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t bits = (uint32_t)((q < 2 ? see0 : see1) >> ((q & 1) * 32));
 #pragma unroll
-          for (int c = 0; c < 32; ++c) mx = fmaxf(mx, ((bits >> c) & 1u) ? __uint_as_float(r[c]) : -CUDART_INF_F);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(r[c]));
+          for (int c = 0; c < 32; ++c)
+            if (!((bits >> c) & 1u)) r[q][c] = 0xFF800000u;            // -inf: exp2 gives an exact 0
         }
       }
+      // row maximum, four independent chains
+      float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mx4[q] = fmaxf(mx4[q], __uint_as_float(r[q][c]));
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float mx_x = mx * a.scale_log2;
       float alpha = 1.f;
       if (m_used == -CUDART_INF_F) m_used = mx_x;
@@ -397,31 +404,24 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       }
       const float m_eff = (m_used == -CUDART_INF_F) ? 0.f : m_used;
 
-      // ---- pass 2: P = exp2(S * scale - max) as bf16 over S; row sum ----
-      float sum = 0.f;
+      // ---- P = exp2(S * scale - max) as bf16 over S; row sum in four chains ----
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t pk[32];
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-          const int c0 = half * 64 + q * 32;
-          uint32_t r[32];
-          tc_ld32(t_S + c0, r);
-          tc_wait_ld();
-          const uint32_t bits = masked ? (uint32_t)((c0 < 64 ? see0 : see1) >> (c0 & 63)) : 0xFFFFFFFFu;
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(r[c]), a.scale_log2, -m_eff));
-            float p1 = fast_exp2(fmaf(__uint_as_float(r[c + 1]), a.scale_log2, -m_eff));
-            if (!((bits >> c) & 1u)) p0 = 0.f;
-            if (!((bits >> (c + 1)) & 1u)) p1 = 0.f;
-            sum += p0 + p1;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(r[half * 2 + q][c]), a.scale_log2, -m_eff));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(r[half * 2 + q][c + 1]), a.scale_log2, -m_eff));
+            sum4[(c >> 1) & 3] += p0 + p1;
             pk[q * 16 + (c >> 1)] = pack_bf16x2(p0, p1);
           }
         }
         tc_st32(t_S + half * 32, pk);
       }
-      l_run += sum;
+      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 
       // ---- rare: the reference maximum moved, rescale the accumulator of this row's warp ----
       if (it > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {

@@ -108,6 +108,7 @@ struct talon_ctx {
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int attn_min_tiles;                // split-KV: key tiles a CTA should at least own
   int pdl;                           // 1: kernels are launched with programmatic stream serialization
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
