@@ -167,6 +167,30 @@ __device__ inline float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed fp32 pairs (sm_100): one instruction for two lanes of a 64-bit register pair.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ inline uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t *>(&v);
@@ -392,7 +416,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
       for (int q = 0; q < 4; ++q)
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mx4[q] = fmaxf(mx4[q], __uint_as_float(r[q][c]));
+        for (int c = 0; c < 32; c += 2) mx4[q] = max3(mx4[q], __uint_as_float(r[q][c]), __uint_as_float(r[q][c + 1]));
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float mx_x = mx * a.scale_log2;
       float alpha = 1.f;
@@ -404,8 +428,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       }
       const float m_eff = (m_used == -CUDART_INF_F) ? 0.f : m_used;
 
-      // ---- P = exp2(S * scale - max) as bf16 over S; row sum in four chains ----
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      // ---- P = exp2(S * scale - max) as bf16 over S; row sum in four packed chains ----
+      const unsigned long long scale2 = pack_f32x2(a.scale_log2, a.scale_log2);
+      const unsigned long long nmax2 = pack_f32x2(-m_eff, -m_eff);
+      unsigned long long sum2[4] = {0ull, 0ull, 0ull, 0ull};          // four pairs of 0.f
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t pk[32];
@@ -413,13 +439,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         for (int q = 0; q < 2; ++q) {
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(r[half * 2 + q][c]), a.scale_log2, -m_eff));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(r[half * 2 + q][c + 1]), a.scale_log2, -m_eff));
-            sum4[(c >> 1) & 3] += p0 + p1;
+            const unsigned long long x2 =
+                fma_f32x2(pack_f32x2(__uint_as_float(r[half * 2 + q][c]), __uint_as_float(r[half * 2 + q][c + 1])), scale2, nmax2);
+            float x0, x1;
+            unpack_f32x2(x2, x0, x1);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            sum2[(c >> 1) & 3] = add_f32x2(sum2[(c >> 1) & 3], pack_f32x2(p0, p1));
             pk[q * 16 + (c >> 1)] = pack_bf16x2(p0, p1);
           }
         }
         tc_st32(t_S + half * 32, pk);
+      }
+      float sum4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float lo, hi;
+        unpack_f32x2(sum2[q], lo, hi);
+        sum4[q] = lo + hi;
       }
       l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 
