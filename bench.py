@@ -421,9 +421,12 @@ def run_talon(args, cfg):
         intensity = att_flops_step / max(1.0, per_step["tree_attention"])
         ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
         bound = "hbm"
+        ratio = roofline.captured_traffic_ratio(dominant)
         roof = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                "traffic": None, "launches_timed": int(dom_n), "avg_launch_us": dom_ms / dom_n * 1e3,
+                "traffic": None if ratio is None else ratio * dom_bytes_total * timed_frac / dom_n,
+                "traffic_source": None if ratio is None else "ncu capture of an earlier run, same kernel source: DRAM bytes per algorithmic byte x this run's bytes per launch",
+                "launches_timed": int(dom_n), "avg_launch_us": dom_ms / dom_n * 1e3,
                 "algorithmic_bytes_per_launch": dom_bytes_total * timed_frac / dom_n}
         if dominant == "tree_attention" and intensity > ridge:
             tf = att_flops_step * K * timed_frac / (dom_ms * 1e-3) / 1e12

@@ -7,6 +7,7 @@ per-chunk top-k lists) is deliberately not counted, so it shows up as lost bandw
 """
 from __future__ import annotations
 
+import hashlib
 import json
 import os
 from typing import Dict, Sequence
@@ -59,3 +60,24 @@ def attention_bytes(prefix_len: int, n_nodes: int, n_q_heads: int, n_kv_heads: i
 
 def attention_flops(prefix_len: int, n_nodes: int, n_q_heads: int, head_dim: int) -> int:
     return 4 * head_dim * n_q_heads * n_nodes * (prefix_len + n_nodes)
+
+
+def captured_traffic_ratio(kernel: str):
+    """DRAM bytes per algorithmic byte of ``kernel`` from its last ncu capture, or None.
+
+    ``traffic_capture.json`` records, per kernel, the ratio measured under ncu together with a
+    hash of the kernel's source files at that time; a kernel whose source changed since then has
+    no valid counters, so None is returned and the benchmark reports ``traffic`` as null."""
+    here = os.path.dirname(os.path.abspath(__file__))
+    try:
+        with open(os.path.join(here, "traffic_capture.json")) as f:
+            rec = json.load(f)[kernel]
+        h = hashlib.sha256()
+        for rel in rec["sources"]:
+            with open(os.path.join(os.path.dirname(here), rel), "rb") as src:
+                h.update(src.read())
+        if h.hexdigest() != rec["sha256"]:
+            return None
+        return float(rec["dram_bytes_per_algorithmic_byte"])
+    except (OSError, KeyError, ValueError):
+        return None
