@@ -256,6 +256,10 @@ enum {
  * the events.  Do not capture a stream into a CUDA graph while timing is on. */
 talon_status talon_timing_enable(talon_ctx *ctx, int32_t max_launches, uint32_t kernel_mask);
 
+/* Suspends (paused != 0) or resumes the bracketing without touching the events, so that a
+ * caller can time a sample of its steps and leave the others undisturbed. */
+talon_status talon_timing_pause(talon_ctx *ctx, int32_t paused);
+
 /* Synchronises `stream`, adds up the elapsed time of the bracketed launches per kernel family
  * since the last read, and makes all pairs available again.
  * ms        host [TALON_N_KERNELS] summed milliseconds

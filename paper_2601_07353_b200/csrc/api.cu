@@ -278,7 +278,14 @@ talon_status talon_timing_enable(talon_ctx *c, int32_t max_launches, uint32_t ke
   for (int i = 0; i < 2 * max_launches; ++i) TALON_CUDA_OK(cudaEventCreate(&c->ev[i]));
   c->ev_cap = max_launches;
   c->ev_used = 0;
+  c->ev_paused = 0;
   c->ev_mask = kernel_mask ? kernel_mask : 0xFFFFFFFFu;
+  return TALON_OK;
+}
+
+talon_status talon_timing_pause(talon_ctx *c, int32_t paused) {
+  if (!c) return TALON_ERR_INVALID_ARG;
+  c->ev_paused = paused ? 1 : 0;
   return TALON_OK;
 }
 

@@ -123,6 +123,7 @@ struct talon_ctx {
   int *ev_kernel;                    // [ev_cap] kernel id of each pair
   int ev_cap, ev_used;
   unsigned ev_mask;                  // kernel families that are timed
+  int ev_paused;                     // 1: launches are not bracketed for now
 };
 
 namespace talon {
@@ -160,7 +161,7 @@ struct LaunchTimer {
   cudaStream_t st;
   int slot;
   LaunchTimer(talon_ctx *ctx, int kernel, cudaStream_t stream) : c(ctx), st(stream), slot(-1) {
-    if (c->ev && ((c->ev_mask >> kernel) & 1u) && c->ev_used < c->ev_cap) {
+    if (c->ev && !c->ev_paused && ((c->ev_mask >> kernel) & 1u) && c->ev_used < c->ev_cap) {
       slot = c->ev_used++;
       c->ev_kernel[slot] = kernel;
       cudaEventRecord(c->ev[2 * slot], st);

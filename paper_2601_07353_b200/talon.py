@@ -52,6 +52,7 @@ _lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
 _lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i64, _i32, _f32, _vp,
                             _vp, _i64] + [_vp] * 5)
 _lib.talon_timing_enable.argtypes = [_vp, _i32, C.c_uint32]
+_lib.talon_timing_pause.argtypes = [_vp, _i32]
 _lib.talon_timing_read.argtypes = [_vp, _vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.talon_kernel_name.argtypes = [_i32]
 _lib.talon_kernel_name.restype = C.c_char_p
@@ -62,12 +63,14 @@ _lib.talon_status_string.argtypes = [C.c_int]
 _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
-           "talon_step", "talon_timing_enable", "talon_timing_read", "talon_target_argmax_noalloc"):
+           "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
+           "talon_target_argmax_noalloc"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
             "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
-            "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_kernel_name",
+            "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
+            "talon_kernel_name",
             "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc"]
 NOALLOC_MAX_ROWS = 8192
 N_KERNELS = 8
@@ -221,6 +224,9 @@ class Talon:
         for k in kernels or ():
             mask |= 1 << KERNEL_NAMES.index(k)
         _check(_lib.talon_timing_enable(self._ctx, max_launches, mask), "talon_timing_enable")
+
+    def timing_pause(self, paused: bool):
+        _check(_lib.talon_timing_pause(self._ctx, 1 if paused else 0), "talon_timing_pause")
 
     def timing_read(self):
         """Returns {kernel name: (summed ms, launches)} since the last read (synchronises the stream)."""
