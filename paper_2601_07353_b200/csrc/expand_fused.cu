@@ -313,16 +313,29 @@ struct TailSmem {
   unsigned char *state;     // [N-1][k]        bit0 eligible, bit2 selected
 };
 
-__device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int row0, int F, int S,
+// Log-sum-exp of a frontier row from its maximum and its sum of exponentials; a row that is not
+// finite flags the sequence.
+__device__ __forceinline__ void finish_row(const FusedArgs &a, const TailSmem &sm, int j, float m, double t,
+                                           int *s_bad) {
+  double lse = (double)m + log(t);
+  if (!(t > 0.0) || !(m < CUDART_INF_F) || lse != lse) {
+    lse = CUDART_NAN;
+    *s_bad = 1;
+    atomicOr(a.status, STATUS_NONFINITE);
+  }
+  sm.row_m[j] = m;
+  sm.row_t[j] = lse;
+  sm.row_cnt[j] = 0;
+}
+
+__device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int lo, int row0, int F, int S,
                             u64 *s_anchor, int *s_cnt, int *s_bad) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = a.k, ks = a.key_stride;
   const int n = a.t.n_nodes[b];
-  const int lo = a.t.layer_off[b * a.lo_stride + a.d];
   const int R = a.N - n;
   const int ke = min(k, R);                 // a parent can place at most R children
   const size_t nb = (size_t)b * a.N;
-  if (tid == 0) { *s_anchor = 0ull; *s_cnt = 0; *s_bad = 0; }
 
   // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys.
   // One warp per row, one lane per chunk (S <= 32). ----
@@ -334,25 +347,48 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
     const size_t item0 = (size_t)row0 * S;
     u64 *st = sm.stage;                           // st[(j * S + c) * k + i]
     const int nkeys = F * S * k;
-    for (int idx = tid; idx < nkeys; idx += EXP_THREADS) {
+    // The compiler cannot move a global load above a store through a shared-memory pointer it
+    // cannot tell apart, so every round of loads goes to registers before anything is stored:
+    // one trip to L2 per round instead of one per load.
+    auto key_at = [&](int idx) {
       const int jc = idx / k, i = idx - jc * k;
-      st[idx] = __ldcg(a.part_keys + (item0 + jc) * ks + i);
+      return __ldcg(a.part_keys + (item0 + jc) * ks + i);
+    };
+    const u64 key_first = tid < nkeys ? key_at(tid) : 0ull;
+    if (tid < F) {
+      const int j = tid;
+      float2 ms[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        ms[c] = c < S ? __ldcg(a.part_ms + item0 + (size_t)j * S + c) : make_float2(-CUDART_INF_F, 0.f);
+      const double ps = a.t.score[nb + lo + j];
+      u64 mk[4];
+#pragma unroll
+      for (int w = 0; w < 4; ++w) mk[w] = w < a.W ? a.t.mask[(nb + lo + j) * a.W + w] : 0ull;
+      float mx = -CUDART_INF_F;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) mx = fmaxf(mx, ms[c].x);
+      double t = 0.0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (ms[c].y != ms[c].y) t += (double)ms[c].y;                     // NaN or +inf logit in the chunk
+        else if (ms[c].x > -CUDART_INF_F) t += (double)ms[c].y * (double)exp2f((ms[c].x - mx) * LOG2E_F);
+      }
+      sm.row_ps[j] = ps;
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        if (w < a.W) sm.row_mask[j * a.W + w] = mk[w];
+      for (int w = 4; w < a.W; ++w) sm.row_mask[j * a.W + w] = a.t.mask[(nb + lo + j) * a.W + w];
+      finish_row(a, sm, j, mx, t, s_bad);
+    }
+    if (tid < nkeys) st[tid] = key_first;
+    for (int idx = tid + EXP_THREADS; idx < nkeys; idx += 2 * EXP_THREADS) {
+      const u64 k0 = key_at(idx);
+      const u64 k1 = idx + EXP_THREADS < nkeys ? key_at(idx + EXP_THREADS) : 0ull;
+      st[idx] = k0;
+      if (idx + EXP_THREADS < nkeys) st[idx + EXP_THREADS] = k1;
     }
     for (int idx = tid; idx < F * k; idx += EXP_THREADS) sm.row_keys[idx] = 0ull;
-    for (int j = tid; j < F; j += EXP_THREADS) {
-      sm.row_ps[j] = a.t.score[nb + lo + j];
-      for (int w = 0; w < a.W; ++w) sm.row_mask[j * a.W + w] = a.t.mask[(nb + lo + j) * a.W + w];
-      float mx = -CUDART_INF_F;
-      for (int c = 0; c < S; ++c) mx = fmaxf(mx, __ldcg(a.part_ms + item0 + (size_t)j * S + c).x);
-      double t = 0.0;
-      for (int c = 0; c < S; ++c) {
-        const float2 ms = __ldcg(a.part_ms + item0 + (size_t)j * S + c);
-        if (ms.y != ms.y) t += (double)ms.y;                              // NaN or +inf logit in the chunk
-        else if (ms.x > -CUDART_INF_F) t += (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
-      }
-      sm.row_m[j] = mx;
-      sm.row_t[j] = t;
-    }
     __syncthreads();
     // a key's rank in its row: its place in its own list plus, for every other chunk of the
     // row, how many of that chunk's keys beat it (keys are unique; lists are descending)
@@ -380,20 +416,32 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
     u64 *st = sm.stage + warp * stage_words;       // st[i * 32 + c] = i-th best key of chunk c
     u64 *sv = st + 32 * k;                         // keys that reach the bound
     u64 *rk = sm.row_keys + (size_t)j * k;
-    // everything this row needs from global memory, issued together
+    // Everything this row needs from global memory goes to registers before the first store
+    // (a load cannot pass a store through a pointer the compiler cannot tell apart): one trip
+    // to L2 for the row, not one per load.
     const float2 ms = (lane < S) ? __ldcg(a.part_ms + item0 + lane) : make_float2(-CUDART_INF_F, 0.f);
+    const double ps = lane == 0 ? a.t.score[nb + lo + j] : 0.0;
+    const u64 pmask = lane < a.W ? a.t.mask[(nb + lo + j) * a.W + lane] : 0ull;
     if (S == 1) {
-      if (lane < k) rk[lane] = __ldcg(a.part_keys + item0 * ks + lane);
-    } else if (lane < S) {
-      const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(a.part_keys + (item0 + lane) * ks);
-      for (int i2 = 0; i2 < ks / 2; ++i2) {        // slots k..ks-1 of a list always hold zero
-        const ulonglong2 x = __ldcg(src + i2);
-        if (2 * i2 < k) st[(2 * i2) * 32 + lane] = x.x;
-        if (2 * i2 + 1 < k) st[(2 * i2 + 1) * 32 + lane] = x.y;
+      const u64 key = lane < k ? __ldcg(a.part_keys + item0 * ks + lane) : 0ull;
+      if (lane < k) rk[lane] = key;
+    } else {
+      const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(a.part_keys + (item0 + min(lane, S - 1)) * ks);
+      for (int i0 = 0; i0 < k; i0 += 16) {         // slots k..ks-1 of a list always hold zero
+        ulonglong2 x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          x[u] = (lane < S && i0 + 2 * u < k) ? __ldcg(src + i0 / 2 + u) : make_ulonglong2(0ull, 0ull);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + 2 * u;
+          if (lane < S && i < k) st[i * 32 + lane] = x[u].x;
+          if (lane < S && i + 1 < k) st[(i + 1) * 32 + lane] = x[u].y;
+        }
       }
     }
-    if (lane == 0) sm.row_ps[j] = a.t.score[nb + lo + j];
-    if (lane < a.W) sm.row_mask[j * a.W + lane] = a.t.mask[(nb + lo + j) * a.W + lane];
+    if (lane == 0) sm.row_ps[j] = ps;
+    if (lane < a.W) sm.row_mask[j * a.W + lane] = pmask;
 
     float mx = ms.x;
 #pragma unroll
@@ -403,7 +451,7 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
     else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
 #pragma unroll
     for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
-    if (lane == 0) { sm.row_m[j] = mx; sm.row_t[j] = t; }
+    if (lane == 0) finish_row(a, sm, j, mx, t, s_bad);
     if (S == 1) continue;
 
     if (lane < k) rk[lane] = 0ull;
@@ -454,20 +502,6 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int r
   }
   __syncthreads();
 
-  // ---- log-sum-exp of every row ----
-  for (int j = tid; j < F; j += EXP_THREADS) {
-    const double t = sm.row_t[j];
-    const float m = sm.row_m[j];
-    double lse = (double)m + log(t);
-    if (!(t > 0.0) || !(m < CUDART_INF_F) || lse != lse) {
-      lse = CUDART_NAN;
-      *s_bad = 1;
-      atomicOr(a.status, STATUS_NONFINITE);
-    }
-    sm.row_t[j] = lse;
-    sm.row_cnt[j] = 0;
-  }
-  __syncthreads();
   if (*s_bad) {            // a frontier row was not finite: this sequence adds nothing
     if (tid == 0) a.t.layer_off[b * a.lo_stride + a.d + 2] = n;
     return;
@@ -974,6 +1008,7 @@ expand_fused_kernel(FusedArgs a) {
     if (tid == 0) {
       s_pool_n = 0;
       s_thr_cta = 0u;
+      s_anchor = 0ull; s_cnt = 0; s_bad = 0;        // the selection phase's accumulators
       cuda::atomic_ref<unsigned int, cuda::thread_scope_device> cnt(a.seq_count[rl.b]);
       const unsigned prev = cnt.fetch_add(1u, cuda::memory_order_acq_rel);
       s_last = (prev == (unsigned)(rl.F * g.splits) - 1u);
@@ -994,7 +1029,7 @@ expand_fused_kernel(FusedArgs a) {
     sm.row_cnt = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
     sm.row_off = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
     sm.state = p;
-    select_tail(a, sm, rl.b, rl.row0, rl.F, g.splits, &s_anchor, &s_cnt, &s_bad);
+    select_tail(a, sm, rl.b, rl.node - rl.j, rl.row0, rl.F, g.splits, &s_anchor, &s_cnt, &s_bad);
     __syncthreads();     // the next chunk's bulk copies land in the memory the selection phase just used
   }
 }
