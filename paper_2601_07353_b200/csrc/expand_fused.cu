@@ -305,7 +305,7 @@ struct TailSmem {
   u64 *stage;        // [EXP_WARPS][32 k + FX_SURV]  chunk lists of the row a warp is merging, survivors
   u64 *row_keys;     // [N-1][k]               per-row top-k keys, descending
   double *score;     // [N-1][k]               log p(u) of each pooled candidate
-  double *row_t;     // [N-1]                  sum of exponentials, then the row's log-sum-exp
+  double *row_t;     // [N-1]                  sum of exponentials relative to row_m
   double *row_ps;    // [N-1]                  log p(v) of the row's parent
   u64 *row_mask;     // [N-1][W]               ancestor mask of the row's parent
   float *row_m;      // [N-1]
@@ -313,18 +313,18 @@ struct TailSmem {
   unsigned char *state;     // [N-1][k]        bit0 eligible, bit2 selected
 };
 
-// Log-sum-exp of a frontier row from its maximum and its sum of exponentials; a row that is not
-// finite flags the sequence.
+// Leaves a frontier row's maximum m and sum of exponentials t for the scoring phase, which takes
+// the logarithm once per candidate, in parallel (one thread taking it here would hold up its whole
+// warp).  m + log t is a finite number exactly when m is finite and 0 < t < inf; anything else
+// (a NaN or +inf logit, a row of -inf only) flags the sequence.
 __device__ __forceinline__ void finish_row(const FusedArgs &a, const TailSmem &sm, int j, float m, double t,
                                            int *s_bad) {
-  double lse = (double)m + log(t);
-  if (!(t > 0.0) || !(m < CUDART_INF_F) || lse != lse) {
-    lse = CUDART_NAN;
+  if (!(t > 0.0) || !(t < CUDART_INF) || !(m < CUDART_INF_F) || !(m > -CUDART_INF_F)) {
     *s_bad = 1;
     atomicOr(a.status, STATUS_NONFINITE);
   }
   sm.row_m[j] = m;
-  sm.row_t[j] = lse;
+  sm.row_t[j] = t;
   sm.row_cnt[j] = 0;
 }
 
@@ -513,7 +513,7 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int l
     const int j = c / k, i = c - j * k;
     const u64 key = sm.row_keys[c];
     double s = -CUDART_INF;
-    if (i < ke && key != 0ull) s = sm.row_ps[j] + ((double)key_logit(key) - sm.row_t[j]);
+    if (i < ke && key != 0ull) s = sm.row_ps[j] + ((double)key_logit(key) - ((double)sm.row_m[j] + log(sm.row_t[j])));
     const bool ok = (s > -CUDART_INF) && (s == s);
     if (!ok) s = -CUDART_INF;
     sm.score[c] = s;
@@ -859,30 +859,20 @@ expand_fused_kernel(FusedArgs a) {
       float tau = lane < EXP_THREADS / grp ? s_gmax[lane] : CUDART_INF_F;
 #pragma unroll
       for (int o = 16; o; o >>= 1) tau = fminf(tau, __shfl_xor_sync(FULL, tau, o));
-      int mine = 0;
-#pragma unroll
-      for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-        for (int e = 0; e < EXP_VEC; ++e)
-          mine += (v[u][e] >= tau && start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
-      int inc = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(FULL, inc, o);
-        if (lane >= o) inc += t;
-      }
-      const int total = __shfl_sync(FULL, inc, 31);
-      int pos = 0;
-      if (lane == 0 && total > 0) pos = atomicAdd(&s_pool_n, total);
-      pos = __shfl_sync(FULL, pos, 0) + inc - mine;
-      if (mine > 0 && pos + mine <= FX_POOL) {
+      // Only a thread whose own maximum reaches the bound holds candidates (about 8 H(8) = 22 of
+      // the 256 do): those append to the CTA's pool themselves.  -inf never competes (probability
+      // zero, and it is what the slots past `end` hold), so the bound is kept finite.
+      const float tau_f = fmaxf(tau, -CUDART_MAX_NORMAL_F);
+      if (bm >= tau_f) {
 #pragma unroll
         for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) {
-            const int tok = start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-            if (v[u][e] >= tau && tok < end) s_pool[pos++] = cand_key(v[u][e], (uint32_t)tok);
-          }
+          for (int e = 0; e < EXP_VEC; ++e)
+            if (v[u][e] >= tau_f) {
+              const int pos = atomicAdd(&s_pool_n, 1);
+              if (pos < FX_POOL)
+                s_pool[pos] = cand_key(v[u][e], (uint32_t)(start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e));
+            }
       }
       __syncthreads();
       if (s_pool_n > FX_POOL) {
