@@ -18,6 +18,14 @@ What follows which passage:
 * ``target_argmax`` / ``accept`` -- Appendix B steps (1)-(2) at temperature 0: the longest
   root-to-leaf prefix whose tokens equal the target's greedy choices, plus the target's
   token at the point of divergence.
+* ``accept_stochastic``          -- Appendix B steps (1)-(3) under sampling (the paper's
+  temperature-1 setting): the target's posterior at each visited node, the children of
+  that node tried one after the other as proposals, and on rejection of all of them a
+  correction token drawn from what is left of the posterior.  The appendix names the three
+  steps and the property they must have (the emitted tokens are distributed exactly as the
+  target model's) and leaves the procedure to the tree-verification literature it cites; the
+  procedure written here is the recursive rejection scheme of that literature for proposals
+  that are fixed rather than sampled, and the property is what pins it.
 
 Readings taken where the paper is silent (all listed in the design notes): the budget N
 counts the root; ``max_depth`` is an extra stop; a per-parent candidate cap ``cand_topk``
@@ -269,3 +277,58 @@ def accept(tree: Tree, t: np.ndarray):
         path.append(nxt)
         cur = nxt
     return len(path) - 1, path, int(t[cur])
+
+
+def children_of(tree: Tree, node: int) -> List[int]:
+    """Children of ``node`` in storage order (ascending token id within a parent)."""
+    return [c for c in range(tree.n_nodes) if tree.parent[c] == node]
+
+
+def target_posterior(z32: np.ndarray, temperature: float = 1.0) -> np.ndarray:
+    """Appendix B step (1): softmax(z / T) of one target-logit row, in fp64."""
+    z = np.asarray(z32, dtype=np.float64) / float(temperature)
+    if np.isnan(z).any() or np.isposinf(z).any() or not np.isfinite(z.max()):
+        raise NonFiniteLogits("target row has no softmax")
+    e = np.exp(z - z.max())
+    return e / e.sum()
+
+
+def accept_stochastic(tree: Tree, target_logits: np.ndarray, u_accept: np.ndarray, u_sample: float,
+                      temperature: float = 1.0):
+    """Sampling verification (Appendix B steps 1-3).
+
+    At the current node (the root first) let p be the target's posterior there.  Its children
+    are proposals that were fixed by the draft tree, not drawn, so each is a proposal
+    distribution with all its mass on one token: child c with token w is accepted with
+    probability p(w) / (mass still unclaimed), decided by the uniform ``u_accept[c]``; a rejected
+    child's token is struck from p.  The first accepted child becomes the current node.  When
+    every child of the current node is rejected (or it has none), the correction token is drawn
+    from what is left of p by inverse CDF in token order with ``u_sample``.  Returns
+    (accept_len, accepted node indices incl. root, correction token).
+
+    The uniforms lie in [0, 1) and come from the caller: node c consumes ``u_accept[c]`` at most
+    once (it has one parent), the sequence consumes ``u_sample`` once.
+    """
+    cur = 0
+    path = [0]
+    while True:
+        p = target_posterior(target_logits[cur], temperature)
+        mass = 1.0
+        nxt = -1
+        for c in children_of(tree, cur):
+            w = int(tree.token[c])
+            if float(u_accept[c]) * mass < p[w]:
+                nxt = c
+                break
+            mass -= p[w]
+            p[w] = 0.0
+        if nxt < 0:
+            break
+        path.append(nxt)
+        cur = nxt
+    cdf = np.cumsum(p)
+    total = cdf[-1]
+    tok = int(np.searchsorted(cdf, float(u_sample) * total, side="right"))
+    last = int(np.nonzero(p > 0.0)[0][-1])           # rounding at u -> 1 must not leave the support
+    tok = min(tok, last)
+    return len(path) - 1, path, tok
