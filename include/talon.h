@@ -164,6 +164,29 @@ talon_status talon_accept(talon_ctx *ctx, const talon_tree *tree, const float *t
                           int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                           int32_t *accept_nodes, int32_t *bonus_tok, void *stream);
 
+/* Sampling verification (Appendix B steps 1-3, the paper's temperature-1 setting; the appendix
+ * names the steps and the property -- what is emitted is distributed exactly as the target
+ * model's own samples -- and leaves the procedure to the literature it cites).  With p the
+ * target's posterior softmax(target_logits / temperature) after the current node (the root
+ * first), the children of that node are tried in storage order: child c with token w is
+ * accepted when u_accept[c] * (mass not yet struck) < p(w), otherwise w is struck from p.  The
+ * first accepted child becomes the current node; when none is accepted the correction token is
+ * drawn from what is left of p by inverse CDF in token order with u_sample.
+ * target_logits device fp32, row of node i of sequence b at (b*N + i) * row_stride; 16-byte aligned rows
+ * temperature   host value, > 0
+ * u_accept      device [B, N] fp64 uniforms in [0, 1): node c consumes u_accept[b, c] if it is tried
+ * u_sample      device [B] fp64 uniforms in [0, 1)
+ * accept_len    device [B]; accept_nodes device [B, D_max + 1] (root first, -1 padded)
+ * out_tok       device [B]: the correction token (the bonus token when a leaf was reached)
+ * Vocabularies above 262144 return TALON_ERR_UNSUPPORTED.  A row without a softmax (NaN, +inf,
+ * only -inf) sets the NONFINITE status; that sequence gets accept_len 0 and out_tok -1.
+ * Decisions are taken in fp64 from fp32 row statistics: a uniform within about 1e-6 (relative) of
+ * its threshold may fall on the other side than in exact arithmetic. */
+talon_status talon_accept_sample(talon_ctx *ctx, const talon_tree *tree, const float *target_logits,
+                                 int64_t row_stride, double temperature, const double *u_accept,
+                                 const double *u_sample, int32_t *accept_len, int32_t *accept_nodes,
+                                 int32_t *out_tok, void *stream);
+
 /* Synchronises `stream`, reads and returns the device status word (OK, NONFINITE, TIMEOUT,
  * CAPACITY).  The word stays set until the next talon_reset. */
 talon_status talon_poll_status(talon_ctx *ctx, void *stream);
@@ -246,7 +269,9 @@ enum {
   TALON_K_COMBINE = 5,      /* merge of split-KV partials                                   */
   TALON_K_ARGMAX = 6,       /* target argmax                                                */
   TALON_K_WALK = 7,         /* greedy accept walk                                           */
-  TALON_N_KERNELS = 8
+  TALON_K_ROWSTATS = 8,     /* softmax normaliser of the target rows (sampling verification) */
+  TALON_K_SAMPLE = 9,       /* rejection walk and correction-token draw                     */
+  TALON_N_KERNELS = 10
 };
 
 /* Per-kernel device timing.  With max_launches > 0 the context creates that many pairs of

@@ -139,6 +139,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
   alloc((void **)&c->d_seq_count, sizeof(unsigned int) * (size_t)p->batch_max);
   alloc((void **)&c->d_argmax, sizeof(unsigned long long) * nrow);
   alloc((void **)&c->d_target_tok, sizeof(int32_t) * nrow);
+  alloc((void **)&c->d_samp_ms, sizeof(float2) * nrow * talon::EXP_MAX_SPLITS);
   c->attn_o_elems = talon::attention_workspace_elems(c, &c->attn_ml_elems);
   alloc((void **)&c->d_attn_o, sizeof(float) * c->attn_o_elems);
   alloc((void **)&c->d_attn_ml, sizeof(float2) * c->attn_ml_elems);
@@ -166,7 +167,7 @@ talon_status talon_destroy(talon_ctx *c) {
   cudaSetDevice(c->device);
   cudaFree(c->d_status); cudaFree(c->d_prefix_len); cudaFree(c->d_part_keys); cudaFree(c->d_part_ms);
   cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_seq_count); cudaFree(c->d_argmax);
-  cudaFree(c->d_target_tok); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
+  cudaFree(c->d_target_tok); cudaFree(c->d_samp_ms); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
   talon_timing_enable(c, 0, 0u);
   delete c;
@@ -234,6 +235,17 @@ talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target
                               (cudaStream_t)stream);
 }
 
+talon_status talon_accept_sample(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                                 double temperature, const double *u_accept, const double *u_sample,
+                                 int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, void *stream) {
+  if (!c || !tree_complete(t) || !target_logits || !u_accept || !u_sample || !accept_len || !accept_nodes || !out_tok)
+    return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || !(temperature > 0.0) || !std::isfinite(temperature)) return TALON_ERR_INVALID_ARG;
+  if (row_stride < c->p.vocab || (row_stride & 3) || !aligned16(target_logits)) return TALON_ERR_INVALID_ARG;
+  return talon::launch_accept_sample(c, t, target_logits, row_stride, temperature, u_accept, u_sample, accept_len,
+                                     accept_nodes, out_tok, (cudaStream_t)stream);
+}
+
 talon_status talon_poll_status(talon_ctx *c, void *stream) {
   if (!c) return TALON_ERR_INVALID_ARG;
   int word = 0;
@@ -257,6 +269,8 @@ const char *talon_kernel_name(int32_t k) {
     case TALON_K_COMBINE: return "attention_combine";
     case TALON_K_ARGMAX: return "target_argmax";
     case TALON_K_WALK: return "accept_walk";
+    case TALON_K_ROWSTATS: return "target_softmax_stats";
+    case TALON_K_SAMPLE: return "accept_sample";
   }
   return "unknown";
 }

@@ -113,6 +113,7 @@ struct talon_ctx {
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
   int32_t *d_target_tok;             // [batch_max * N]
+  float2 *d_samp_ms;                 // [batch_max * N, EXP_MAX_SPLITS] per-chunk (max, sum) of target rows
   float *d_attn_o;                   // split-KV partial outputs
   float2 *d_attn_ml;                 // split-KV partial (max, sum)
   size_t attn_o_elems, attn_ml_elems;
@@ -190,6 +191,9 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                            int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st);
+talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                                  double temperature, const double *u_accept, const double *u_sample,
+                                  int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, cudaStream_t st);
 size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems);
 talon_status expand_fused_setup(talon_ctx *c);
 talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,

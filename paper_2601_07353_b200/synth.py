@@ -40,6 +40,8 @@ STREAM_KT = 8
 STREAM_VT = 9
 STREAM_PREFIX = 10
 STREAM_ZIPF = 11
+STREAM_UACCEPT = 12
+STREAM_USAMPLE = 13
 
 DEFAULT_SEED = 20260107
 
@@ -93,6 +95,15 @@ def row_key(seed: int, stream: int, seq_id: int, path_hash: int = 0) -> int:
 def uniform01(key: int) -> float:
     """One uniform in (0,1) with 53 bits, from a key (host scalar)."""
     return ((mix64(key) >> 11) + 0.5) * (1.0 / (1 << 53))
+
+
+def verify_uniforms(seed: int, seq_id: int, n: int, draw: int = 0):
+    """The uniforms a sampling verification of one sequence consumes: one per tree node (NumPy
+    fp64 array of length ``n``) and one for the correction token, all in (0, 1) with 53 bits.
+    ``draw`` numbers independent repetitions."""
+    ku = row_key(seed, STREAM_UACCEPT, seq_id, draw)
+    u = np.array([uniform01((ku + i * _ODD_A) & _M64) for i in range(n)], dtype=np.float64)
+    return u, uniform01(row_key(seed, STREAM_USAMPLE, seq_id, draw))
 
 
 def _arange64(n: int, device=None, start: int = 0):

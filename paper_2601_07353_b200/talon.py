@@ -47,6 +47,7 @@ _lib.talon_layers_run.argtypes = [_vp]
 _lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
 _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.talon_accept_sample.argtypes = [_vp, _TP, _vp, _i64, C.c_double, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_poll_status.argtypes = [_vp, _vp]
 _lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
 _lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i64, _i32, _f32, _vp,
@@ -64,16 +65,16 @@ _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
            "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
-           "talon_target_argmax_noalloc"):
+           "talon_target_argmax_noalloc", "talon_accept_sample"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
             "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
             "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
             "talon_kernel_name",
-            "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc"]
+            "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample"]
 NOALLOC_MAX_ROWS = 8192
-N_KERNELS = 8
+N_KERNELS = 10
 KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
 
 
@@ -199,6 +200,16 @@ class Talon:
         _check(_lib.talon_accept(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, _ptr(target_tok),
                                  _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok), _stream(self.device)),
                "talon_accept")
+
+    def accept_sample(self, tree: Tree, target_logits, temperature: float, u_accept, u_sample, accept_len,
+                      accept_nodes, out_tok, row_stride: Optional[int] = None):
+        ts = tree.struct()
+        if row_stride is None:
+            row_stride = target_logits.stride(-2)
+        assert u_accept.dtype == torch.float64 and u_sample.dtype == torch.float64
+        _check(_lib.talon_accept_sample(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, float(temperature),
+                                        _ptr(u_accept), _ptr(u_sample), _ptr(accept_len), _ptr(accept_nodes),
+                                        _ptr(out_tok), _stream(self.device)), "talon_accept_sample")
 
     def poll_status(self) -> int:
         return _lib.talon_poll_status(self._ctx, _stream(self.device))

@@ -97,3 +97,62 @@ def oracle_tree_from_arrays(g: dict, budget: int, max_depth: int) -> O.Tree:
         t.mask[i, i // 64] |= np.uint64(1) << np.uint64(i % 64)
     t.n_nodes = n
     return t
+
+
+SAMPLE_EPS = 1e-6
+sample_log: List[str] = []       # every tolerated sampling decision, for the test report
+
+
+def follow_sampling(tree: O.Tree, rows, u_accept, u_sample: float, temperature: float, g_len: int, g_path,
+                    g_tok: int, label: str) -> int:
+    """Checks a sampling verification the GPU produced against the oracle's procedure, decision by
+    decision along the GPU's path.  The GPU decides in fp64 from fp32 row statistics, so a decision
+    whose two sides differ by less than SAMPLE_EPS (relative) may fall either way: such a decision is
+    logged and counted, anything else must agree.  Returns the number of tolerated decisions; when it
+    is 0 the GPU result equals ``O.accept_stochastic`` outright (checked too)."""
+    tolerated = 0
+    cur = 0
+    assert int(g_path[0]) == 0, f"{label}: path does not start at the root"
+    step = 0
+    while True:
+        p = O.target_posterior(rows[cur], temperature)
+        mass = 1.0
+        nxt = -1
+        g_next = int(g_path[step + 1]) if step < g_len else -1
+        for c in O.children_of(tree, cur):
+            w = int(tree.token[c])
+            lhs = float(u_accept[c]) * mass
+            take = lhs < p[w]
+            g_take = (c == g_next)
+            if take != g_take:
+                assert abs(lhs - p[w]) <= SAMPLE_EPS * max(p[w], lhs), \
+                    f"{label}: node {cur} child {c}: accept decision differs (u*mass {lhs}, p {p[w]})"
+                tolerated += 1
+                sample_log.append(f"{label}: accept decision at child {c}")
+                take = g_take
+            if take:
+                nxt = c
+                break
+            mass -= p[w]
+            p[w] = 0.0
+        assert nxt == g_next, f"{label}: after node {cur} the GPU went to {g_next}, the procedure to {nxt}"
+        if nxt < 0:
+            break
+        cur = nxt
+        step += 1
+    assert step == g_len, f"{label}: accepted length {g_len} vs {step}"
+    cdf = np.cumsum(p)
+    total = cdf[-1]
+    target = float(u_sample) * total
+    want = min(int(np.searchsorted(cdf, target, side="right")), int(np.nonzero(p > 0.0)[0][-1]))
+    if g_tok != want:
+        assert 0 <= g_tok < len(p) and p[g_tok] > 0.0, f"{label}: correction token {g_tok} has no mass"
+        lo, hi = cdf[g_tok] - p[g_tok], cdf[g_tok]
+        tol = SAMPLE_EPS * total
+        assert lo - tol <= target <= hi + tol, f"{label}: correction token {g_tok} vs {want} beyond tolerance"
+        tolerated += 1
+        sample_log.append(f"{label}: correction token {g_tok} vs {want}")
+    if tolerated == 0:
+        alen, path, tok = O.accept_stochastic(tree, rows, u_accept, u_sample, temperature)
+        assert (alen, path, tok) == (g_len, [int(x) for x in g_path[: g_len + 1]], g_tok), label
+    return tolerated
