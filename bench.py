@@ -365,6 +365,39 @@ def run_talon(args, cfg):
             graph_info = {"error": str(e).splitlines()[0][:200]}
             torch.cuda.synchronize()
 
+    # ---- the sampling verification (the paper's temperature-1 setting) on the same trees: an extra, not the headline ----
+    sampling = None
+    if not args.no_sampling:
+        Ks = min(K, 64)
+        dev_t = sets[0].target.device
+        uas = [torch.from_numpy(np.stack([synth.verify_uniforms(args.seed, sid, N, 0)[0] for sid in wl.seq_ids])).to(dev_t)
+               for wl in sets]
+        uss = [torch.tensor([synth.verify_uniforms(args.seed, sid, N, 0)[1] for sid in wl.seq_ids], dtype=torch.float64,
+                            device=dev_t) for wl in sets]
+        s_tok = torch.zeros(B, dtype=torch.int32, device=dev_t)
+
+        def sample_step(i):
+            wl = sets[i % n_sets]
+            t.accept_sample(wl.tree, wl.target, 1.0, uas[i % n_sets], uss[i % n_sets], wl.accept_len, wl.accept_nodes, s_tok)
+
+        for i in range(3):
+            sample_step(i)
+        torch.cuda.synchronize()
+        t.timing_enable(2 * Ks + 8, ["target_softmax_stats", "accept_sample"])
+        for i in range(Ks):
+            sample_step(i)
+        st = t.timing_read()
+        t.timing_enable(0)
+        assert t.poll_status() == talon.OK
+        sm_ms, sm_n = st["target_softmax_stats"]
+        wk_ms, wk_n = st["accept_sample"]
+        if sm_n and wk_n:
+            gbs = per_step["target_argmax"] / (sm_ms / sm_n * 1e-3) / 1e9
+            sampling = {"temperature": 1.0, "calls": Ks,
+                        "target_softmax_stats": {"ms_per_call": sm_ms / sm_n, "algorithmic_gbs": gbs,
+                                                 "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]},
+                        "accept_sample": {"ms_per_call": wk_ms / wk_n}}
+
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----
     e2e = None
     if not args.no_e2e:
@@ -463,7 +496,7 @@ def run_talon(args, cfg):
                        "step": f"talon_step: reset + {D} expand-layer calls + build + tree attention + accept",
                        "sequences_per_rank": B, "input_sets": n_sets},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "cpu_baseline": cpu,
-            "graph_replay": graph_info, "kernels": kernels,
+            "graph_replay": graph_info, "kernels": kernels, "sampling_verify": sampling,
             "tree_shapes": {"n_nodes_min": min(nn), "n_nodes_max": max(nn), "max_depth_min": min(dp), "max_depth_max": max(dp),
                             "expanded_rows_per_seq_mean": float(np.mean([s[2] for s in shapes]))},
             "sequence_steps_per_s": value * B,
@@ -487,6 +520,7 @@ def main(argv=None):
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sampling", action="store_true", help="skip the sampling-verification extra")
     args = ap.parse_args(argv)
     from paper_2601_07353_b200 import synth
     if args.seed is None:

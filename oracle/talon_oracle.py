@@ -26,6 +26,12 @@ What follows which passage:
   target model's) and leaves the procedure to the tree-verification literature it cites; the
   procedure written here is the recursive rejection scheme of that literature for proposals
   that are fixed rather than sampled, and the property is what pins it.
+* ``commit`` / ``draft_efficiency`` / ``speedup`` -- the bookkeeping either side of one
+  draft-and-verify step in the generation loop of Section 5.3: the accepted tokens' keys and
+  values join the prefix cache, the correction token becomes the next root, and the counts
+  N_p (verification passes), N_q (draft passes) and L (tokens produced) feed the draft
+  efficiency delta = N_q / N_p, the mean accepted tokens tau = L / N_p and the speed-up
+  R = tau / (1 + c delta) of Section 5.3 and its derivation in the appendix.
 
 Readings taken where the paper is silent (all listed in the design notes): the budget N
 counts the root; ``max_depth`` is an extra stop; a per-parent candidate cap ``cand_topk``
@@ -332,3 +338,35 @@ def accept_stochastic(tree: Tree, target_logits: np.ndarray, u_accept: np.ndarra
     last = int(np.nonzero(p > 0.0)[0][-1])           # rounding at u -> 1 must not leave the support
     tok = min(tok, last)
     return len(path) - 1, path, tok
+
+
+def commit(tree: Tree, accept_len: int, path: Sequence[int], next_tok: int, k_tree: np.ndarray, v_tree: np.ndarray,
+           k_prefix: np.ndarray, v_prefix: np.ndarray):
+    """What one finished step leaves for the next one (generation loop of Section 5.3).
+
+    The tokens on the accepted path, root first, are now part of the sequence: their key and
+    value rows (``k_tree[node]``, ``[Hkv, Dh]`` each) are appended to the prefix cache in path
+    order.  The next step starts from ``next_tok``.  Returns (k_prefix', v_prefix', next root,
+    counts) with counts = (verification passes, draft passes, tokens produced) of this step:
+    one target pass, one draft pass per expanded layer (Algorithm 2's loop body), and the
+    accepted tokens plus the correction token."""
+    nodes = [int(x) for x in path[: accept_len + 1]]
+    assert nodes[0] == 0 and len(nodes) == accept_len + 1
+    k_new = np.concatenate([k_prefix, k_tree[nodes]], axis=0)
+    v_new = np.concatenate([v_prefix, v_tree[nodes]], axis=0)
+    return k_new, v_new, int(next_tok), (1, int(tree.layers_run), accept_len + 1)
+
+
+def draft_efficiency(n_q: int, n_p: int) -> float:
+    """delta = N_q / N_p: draft passes invested per verification pass (Section 5.3)."""
+    return n_q / n_p
+
+
+def mean_accepted_tokens(length: int, n_p: int) -> float:
+    """tau = L / N_p: tokens produced per verification pass (Section 5.3)."""
+    return length / n_p
+
+
+def speedup(tau: float, delta: float, c: float) -> float:
+    """R = tau / (1 + c delta), c the draft pass's cost relative to the target pass (Section 5.3)."""
+    return tau / (1.0 + c * delta)
