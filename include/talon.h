@@ -187,6 +187,26 @@ talon_status talon_accept_sample(talon_ctx *ctx, const talon_tree *tree, const f
                                  const double *u_sample, int32_t *accept_len, int32_t *accept_nodes,
                                  int32_t *out_tok, void *stream);
 
+/* What a verified step leaves for the next one (the generation loop of Section 5.3): for every
+ * sequence b the key and value rows of the accepted nodes accept_nodes[b, 0 .. accept_len[b]]
+ * (root first) are copied from k_tree / v_tree to the prefix cache at tokens prefix_len[b] ..
+ * prefix_len[b] + accept_len[b] of the sequence's block, prefix_len[b] grows by accept_len[b] + 1,
+ * root_tok[b] becomes next_tok[b] (talon_accept's bonus_tok or talon_accept_sample's out_tok), and
+ * counters[b] advances by (1, draft passes, accept_len[b] + 1): the N_p, N_q and L of Section 5.3,
+ * a draft pass being a layer Algorithm 2 expanded for this sequence.  The next step starts with
+ * talon_reset(root_tok, prefix_len).
+ * All pointers device memory.  k_tree, v_tree [B, N, Hkv, Dh] bf16; k_prefix, v_prefix, kv_start,
+ * kv_tokens, kv_stride_t, kv_stride_h as in talon_tree_attention (written here);
+ * kv_limit  [B] int64 or null: first token offset past the block of sequence b (kv_tokens if null)
+ * prefix_len [B] in/out; root_tok [B] out; counters [B, 3] int64 in/out or null.
+ * A sequence whose block has no room is left as it is and the CAPACITY status is set. */
+talon_status talon_commit(talon_ctx *ctx, const talon_tree *tree, const int32_t *accept_len,
+                          const int32_t *accept_nodes, const int32_t *next_tok, const void *k_tree,
+                          const void *v_tree, void *k_prefix, void *v_prefix, const int64_t *kv_start,
+                          const int64_t *kv_limit, int64_t kv_tokens, int64_t kv_stride_t,
+                          int64_t kv_stride_h, int32_t *prefix_len, int32_t *root_tok,
+                          int64_t *counters, void *stream);
+
 /* Synchronises `stream`, reads and returns the device status word (OK, NONFINITE, TIMEOUT,
  * CAPACITY).  The word stays set until the next talon_reset. */
 talon_status talon_poll_status(talon_ctx *ctx, void *stream);
@@ -271,7 +291,8 @@ enum {
   TALON_K_WALK = 7,         /* greedy accept walk                                           */
   TALON_K_ROWSTATS = 8,     /* softmax normaliser of the target rows (sampling verification) */
   TALON_K_SAMPLE = 9,       /* rejection walk and correction-token draw                     */
-  TALON_N_KERNELS = 10
+  TALON_K_COMMIT = 10,      /* accepted K/V rows into the prefix cache, counters            */
+  TALON_N_KERNELS = 11
 };
 
 /* Per-kernel device timing.  With max_launches > 0 the context creates that many pairs of

@@ -246,6 +246,23 @@ talon_status talon_accept_sample(talon_ctx *c, const talon_tree *t, const float 
                                      accept_nodes, out_tok, (cudaStream_t)stream);
 }
 
+talon_status talon_commit(talon_ctx *c, const talon_tree *t, const int32_t *accept_len, const int32_t *accept_nodes,
+                          const int32_t *next_tok, const void *k_tree, const void *v_tree, void *k_prefix,
+                          void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
+                          int64_t kv_stride_t, int64_t kv_stride_h, int32_t *prefix_len, int32_t *root_tok,
+                          int64_t *counters, void *stream) {
+  if (!c || !tree_complete(t) || !accept_len || !accept_nodes || !next_tok || !k_tree || !v_tree || !k_prefix ||
+      !v_prefix || !kv_start || !prefix_len || !root_tok)
+    return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || kv_tokens < 0 || kv_tokens > 0x7FFFFFFFll) return TALON_ERR_INVALID_ARG;
+  if ((kv_stride_t & 7) || (kv_stride_h & 7) || kv_stride_t < 0 || kv_stride_h < 0) return TALON_ERR_INVALID_ARG;
+  if (!aligned16(k_prefix) || !aligned16(v_prefix) || !aligned16(k_tree) || !aligned16(v_tree))
+    return TALON_ERR_INVALID_ARG;
+  return talon::launch_commit(c, t, accept_len, accept_nodes, next_tok, k_tree, v_tree, k_prefix, v_prefix, kv_start,
+                              kv_limit, kv_tokens, kv_stride_t, kv_stride_h, prefix_len, root_tok, counters,
+                              (cudaStream_t)stream);
+}
+
 talon_status talon_poll_status(talon_ctx *c, void *stream) {
   if (!c) return TALON_ERR_INVALID_ARG;
   int word = 0;
@@ -271,6 +288,7 @@ const char *talon_kernel_name(int32_t k) {
     case TALON_K_WALK: return "accept_walk";
     case TALON_K_ROWSTATS: return "target_softmax_stats";
     case TALON_K_SAMPLE: return "accept_sample";
+    case TALON_K_COMMIT: return "commit";
   }
   return "unknown";
 }

@@ -194,6 +194,11 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
 talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
                                   double temperature, const double *u_accept, const double *u_sample,
                                   int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, cudaStream_t st);
+talon_status launch_commit(talon_ctx *c, const talon_tree *t, const int32_t *accept_len, const int32_t *accept_nodes,
+                           const int32_t *next_tok, const void *k_tree, const void *v_tree, void *k_prefix,
+                           void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
+                           int64_t stride_t, int64_t stride_h, int32_t *prefix_len, int32_t *root_tok,
+                           int64_t *counters, cudaStream_t st);
 size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems);
 talon_status expand_fused_setup(talon_ctx *c);
 talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,

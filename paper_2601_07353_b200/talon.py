@@ -48,6 +48,7 @@ _lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
 _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_accept_sample.argtypes = [_vp, _TP, _vp, _i64, C.c_double, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.talon_commit.argtypes = [_vp, _TP] + [_vp] * 9 + [_i64, _i64, _i64, _vp, _vp, _vp, _vp]
 _lib.talon_poll_status.argtypes = [_vp, _vp]
 _lib.talon_step_host.argtypes = [_vp, _i32] + [_vp] * 9 + [_f32] + [_vp] * 10
 _lib.talon_step.argtypes = ([_vp, _TP, _i32, _vp, _vp, _vp, _i64, _i32] + [_vp] * 6 + [_i64, _i64, _i64, _i32, _f32, _vp,
@@ -65,16 +66,17 @@ _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
            "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
-           "talon_target_argmax_noalloc", "talon_accept_sample"):
+           "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
             "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status",
             "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
             "talon_kernel_name",
-            "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample"]
+            "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample",
+            "talon_commit"]
 NOALLOC_MAX_ROWS = 8192
-N_KERNELS = 10
+N_KERNELS = 11
 KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
 
 
@@ -210,6 +212,14 @@ class Talon:
         _check(_lib.talon_accept_sample(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, float(temperature),
                                         _ptr(u_accept), _ptr(u_sample), _ptr(accept_len), _ptr(accept_nodes),
                                         _ptr(out_tok), _stream(self.device)), "talon_accept_sample")
+
+    def commit(self, tree: Tree, accept_len, accept_nodes, next_tok, k_tree, v_tree, k_prefix, v_prefix, kv_start,
+               kv_limit, kv_tokens, kv_stride_t, kv_stride_h, prefix_len, root_tok, counters=None):
+        ts = tree.struct()
+        _check(_lib.talon_commit(self._ctx, C.byref(ts), _ptr(accept_len), _ptr(accept_nodes), _ptr(next_tok),
+                                 _ptr(k_tree), _ptr(v_tree), _ptr(k_prefix), _ptr(v_prefix), _ptr(kv_start),
+                                 _ptr(kv_limit), kv_tokens, kv_stride_t, kv_stride_h, _ptr(prefix_len), _ptr(root_tok),
+                                 _ptr(counters), _stream(self.device)), "talon_commit")
 
     def poll_status(self) -> int:
         return _lib.talon_poll_status(self._ctx, _stream(self.device))
