@@ -99,6 +99,19 @@ def _stream(device) -> C.c_void_p:
     return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
 
 
+def loop_metrics(counters: torch.Tensor, cost_ratio: float) -> dict:
+    """Section 5.3's figures from the counters ``talon_commit`` keeps ([B, 3] int64: verification
+    passes N_p, draft passes N_q, tokens produced L), summed over the sequences: draft efficiency
+    delta = N_q / N_p, mean accepted tokens tau = L / N_p and the wall-time speed-up
+    R = tau / (1 + c delta) for a draft pass that costs ``cost_ratio`` = c target passes."""
+    n_p, n_q, length = (int(x) for x in counters.sum(dim=0).tolist())
+    if n_p <= 0:
+        raise ValueError("no verification pass has been committed yet")
+    delta, tau = n_q / n_p, length / n_p
+    return {"n_p": n_p, "n_q": n_q, "tokens": length, "delta": delta, "tau": tau,
+            "speedup": tau / (1.0 + cost_ratio * delta)}
+
+
 def target_argmax_noalloc(target_logits: torch.Tensor, target_tok: torch.Tensor) -> None:
     """``talon_target_argmax_noalloc``: greedy target token of every row of ``target_logits``
     ([rows, V] fp32 on the current CUDA device) into ``target_tok`` ([rows] int32), with no context

@@ -53,3 +53,15 @@ def test_speedup_formula_is_the_wall_time_ratio():
     assert O.draft_efficiency((D + 1) * steps, steps) == D + 1
     # free drafting (c = 0) gives R = tau; drafting as costly as verifying gives tau / (1 + delta)
     assert O.speedup(4.0, 9.0, 0.0) == 4.0 and O.speedup(4.0, 9.0, 1.0) == 0.4
+
+
+def test_binding_loop_metrics_agree_with_the_oracle():
+    import torch
+    from paper_2601_07353_b200 import talon
+    counters = torch.tensor([[3, 20, 11], [3, 31, 7], [2, 9, 9]], dtype=torch.int64)
+    m = talon.loop_metrics(counters, 0.05)
+    n_p, n_q, L = 8, 60, 27
+    assert (m["n_p"], m["n_q"], m["tokens"]) == (n_p, n_q, L)
+    assert abs(m["delta"] - O.draft_efficiency(n_q, n_p)) < 1e-15
+    assert abs(m["tau"] - O.mean_accepted_tokens(L, n_p)) < 1e-15
+    assert abs(m["speedup"] - O.speedup(L / n_p, n_q / n_p, 0.05)) < 1e-15
