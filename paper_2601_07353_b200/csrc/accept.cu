@@ -53,17 +53,28 @@ target_argmax_kernel(ArgmaxArgs a) {
           for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
         }
       }
+      // the tile's maximum first (one max per element); only a tile that raises the thread's
+      // maximum, or the thread's first tile, is searched for where that maximum sits
+      float bm = -CUDART_INF_F;
 #pragma unroll
-      for (int u = 0; u < EXP_UNROLL; ++u) {
-        const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
+      for (int u = 0; u < EXP_UNROLL; ++u)
 #pragma unroll
         for (int e = 0; e < EXP_VEC; ++e) {
-          const float x = v[u][e];
-          bad |= (x != x);
-          // strict > keeps the lowest index among equal values; the first in-range element
-          // claims the slot even if it is -inf
-          if (idx + e < end && (x > bestv || besti == 0xFFFFFFFFu)) { bestv = x; besti = (uint32_t)(idx + e); }
+          bad |= (v[u][e] != v[u][e]);
+          bm = fmaxf(bm, v[u][e]);
         }
+      if (bm > bestv || besti == 0xFFFFFFFFu) {
+        // strict > keeps the earlier tile among equal maxima; inside the tile the first match in
+        // (u, e) order is the thread's lowest index; a tile of -inf only still claims its first slot
+        uint32_t first = 0xFFFFFFFFu;
+#pragma unroll
+        for (int u = EXP_UNROLL - 1; u >= 0; --u)
+#pragma unroll
+          for (int e = EXP_VEC - 1; e >= 0; --e) {
+            const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
+            if (idx < end && v[u][e] == bm) first = (uint32_t)idx;
+          }
+        if (first != 0xFFFFFFFFu) { bestv = bm; besti = first; }
       }
     }
     unsigned long long key = (besti == 0xFFFFFFFFu) ? 0ull : cand_key(bestv, besti);
