@@ -95,7 +95,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *params, int d
 /* Frees the context's workspace.  Caller memory is untouched.  Null is accepted. */
 talon_status talon_destroy(talon_ctx *ctx);
 
-/* Algorithm 2, lines 1-2: T <- {x_t}, P_0 <- {x_t}, p(x_t) <- 1, d <- 0, for B sequences.
+/* Initialisation of Algorithm 2: T <- {x_t}, P_0 <- {x_t}, p(x_t) <- 1, d <- 0, for B sequences.
  * root_tok   device [B]  last committed token x_t of each sequence
  * prefix_len device [B]  number of tokens before x_t, i.e. the KV-cache length L_b (>= 0)
  * Clears the device status word. */
@@ -281,7 +281,7 @@ int64_t talon_launch_count(const talon_ctx *ctx);
 
 /* Kernel families of the library, for talon_timing_read. */
 enum {
-  TALON_K_RESET = 0,        /* tree initialisation (Algorithm 2, lines 1-2)                  */
+  TALON_K_RESET = 0,        /* tree initialisation of Algorithm 2                              */
   TALON_K_EXPAND_ROWS = 1,  /* softmax normaliser + per-parent top-k over the logit rows    */
   TALON_K_SELECT = 2,       /* Top-K / gate / budget truncation / append                    */
   TALON_K_BUILD = 3,        /* positions and sentinels                                      */

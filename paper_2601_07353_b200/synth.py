@@ -11,7 +11,7 @@ case the same integer recipe runs through torch ops on that device.
 
 Workload shapes follow the paper's setting (vocabularies of 32K/128K/152K, node budget
 60, width K <= 10; Section 6 "setup" and the tree-construction micro-benchmark in the
-appendix) and the five benchmark configurations of this build.
+appendix) and five benchmark configurations.
 """
 from __future__ import annotations
 
