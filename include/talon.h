@@ -242,7 +242,13 @@ talon_status talon_step_host(talon_ctx *ctx, int32_t B, const int32_t *root_tok,
  * (q .. out), talon_accept (target_logits .. bonus_tok; target_tok may be null).
  * n_layers  expansion layers to enqueue, 0..D_max (layers after the tree is full cost one
  *           frontier check each and read no logits)
- * Enqueues only; no synchronisation. */
+ * Enqueues only; no synchronisation.
+ * A step is a chain of small dependent kernels, so from the second call with exactly the same
+ * arguments the library captures these launches into a CUDA graph once and replays it on later
+ * calls (same kernels, same memory, one submission; up to 64 argument sets are kept, least
+ * recently used first out).  The plain launch sequence is used on the legacy default stream, while
+ * `stream` is being captured by the caller, while launches are timed (talon_timing_enable without
+ * pause), and always when the environment has TALON_STEP_GRAPH=0. */
 talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const int32_t *root_tok,
                         const int32_t *prefix_len, const float *draft_logits,
                         int64_t draft_row_stride, int32_t n_layers, const void *q,

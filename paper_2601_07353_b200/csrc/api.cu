@@ -118,6 +118,8 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     if (c->attn_min_tiles < 1) c->attn_min_tiles = 1;
     const char *e = std::getenv("TALON_PDL");
     c->pdl = (e && e[0] == '1') ? 1 : 0;
+    const char *g = std::getenv("TALON_STEP_GRAPH");
+    c->step_graph = (g && g[0] == '0') ? 0 : 1;
   }
   c->exp_grid = c->sm_count * talon::EXP_CTAS_PER_SM;
   c->rows_cap = p->batch_max * (p->budget - 1);
@@ -170,6 +172,11 @@ talon_status talon_destroy(talon_ctx *c) {
   cudaFree(c->d_target_tok); cudaFree(c->d_samp_ms); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
   talon_timing_enable(c, 0, 0u);
+  if (c->graphs) {
+    for (int i = 0; i < talon::STEP_GRAPH_SLOTS; ++i)
+      if (c->graphs[i].exec) cudaGraphExecDestroy(c->graphs[i].exec);
+    delete[] c->graphs;
+  }
   delete c;
   return TALON_OK;
 }
@@ -336,15 +343,15 @@ talon_status talon_timing_read(talon_ctx *c, void *stream, double *ms, int64_t *
   return TALON_OK;
 }
 
-talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
-                        const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
-                        int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
-                        const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
-                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
-                        const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
-                        int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok, void *stream) {
-  if (!c) return TALON_ERR_INVALID_ARG;
-  if (n_layers < 0 || n_layers > c->p.max_depth) return TALON_ERR_INVALID_ARG;
+// The launches of one step, in order, on `stream`.
+static talon_status step_enqueue(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
+                                 const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
+                                 int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
+                                 const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
+                                 int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale,
+                                 void *out, const float *target_logits, int64_t target_row_stride,
+                                 int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                                 void *stream) {
   talon_status r = talon_reset(c, t, root_tok, prefix_len, B, stream);
   for (int d = 0; r == TALON_OK && d < n_layers; ++d)
     r = talon_expand_layer(c, t, draft_logits, draft_row_stride, c->p.budget, TALON_ROWS_BY_NODE, stream);
@@ -356,6 +363,102 @@ talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int3
     r = talon_accept(c, t, target_logits, target_row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
                      stream);
   return r;
+}
+
+talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
+                        const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
+                        int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
+                        const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
+                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const float *target_logits, int64_t target_row_stride, int32_t *target_tok,
+                        int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok, void *stream) {
+  if (!c) return TALON_ERR_INVALID_ARG;
+  if (n_layers < 0 || n_layers > c->p.max_depth) return TALON_ERR_INVALID_ARG;
+#define TALON_STEP_ARGS                                                                                              \
+  c, t, B, root_tok, prefix_len, draft_logits, draft_row_stride, n_layers, q, k_prefix, v_prefix, k_tree, v_tree,    \
+      kv_start, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out, target_logits, target_row_stride, \
+      target_tok, accept_len, accept_nodes, bonus_tok, stream
+  cudaStream_t st = (cudaStream_t)stream;
+  // A step is a chain of small dependent kernels, so a caller that repeats it pays mostly for
+  // launches.  From the second call with the very same arguments the launches are captured once
+  // into a CUDA graph and replayed from then on: the same kernels on the same memory, one
+  // submission.  Not on the legacy default stream (it cannot be captured), not while the stream is
+  // already being captured by the caller, and not while launches are being timed with events.
+  const bool timing = c->ev && !c->ev_paused;
+  if (!c->step_graph || !t || st == nullptr || st == cudaStreamLegacy || timing) return step_enqueue(TALON_STEP_ARGS);
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+    cudaGetLastError();
+    return step_enqueue(TALON_STEP_ARGS);
+  }
+  if (!c->graphs) {
+    c->graphs = new (std::nothrow) talon::StepGraph[talon::STEP_GRAPH_SLOTS];
+    if (!c->graphs) return step_enqueue(TALON_STEP_ARGS);
+    std::memset(c->graphs, 0, sizeof(talon::StepGraph) * talon::STEP_GRAPH_SLOTS);
+  }
+  unsigned long long key[talon::STEP_GRAPH_WORDS];
+  std::memset(key, 0, sizeof(key));
+  {
+    int n = 0;
+    auto put = [&](const void *p) { key[n++] = (unsigned long long)reinterpret_cast<uintptr_t>(p); };
+    auto puti = [&](long long v) { key[n++] = (unsigned long long)v; };
+    put(t->n_nodes); put(t->token); put(t->parent); put(t->depth); put(t->position); put(t->layer_off);
+    put(t->score); put(t->mask);
+    puti(B); put(root_tok); put(prefix_len); put(draft_logits); puti(draft_row_stride); puti(n_layers);
+    put(q); put(k_prefix); put(v_prefix); put(k_tree); put(v_tree); put(kv_start); puti(kv_tokens);
+    puti(kv_stride_t); puti(kv_stride_h); puti(max_prefix_len);
+    unsigned int bits; std::memcpy(&bits, &sm_scale, 4); puti(bits);
+    put(out); put(target_logits); puti(target_row_stride); put(target_tok); put(accept_len); put(accept_nodes);
+    put(bonus_tok); put(stream);
+  }
+  talon::StepGraph *hit = nullptr, *victim = &c->graphs[0];
+  for (int i = 0; i < talon::STEP_GRAPH_SLOTS; ++i) {
+    talon::StepGraph *g = &c->graphs[i];
+    if (g->used && std::memcmp(g->args, key, sizeof(key)) == 0) { hit = g; break; }
+    if (!g->used || (victim->used && g->last_use < victim->last_use)) victim = g;
+  }
+  c->step_tick += 1;
+  if (!hit) {                      // first sighting: remember the arguments, run the plain way
+    if (victim->exec) cudaGraphExecDestroy(victim->exec);
+    std::memset(victim, 0, sizeof(*victim));
+    std::memcpy(victim->args, key, sizeof(key));
+    victim->used = true;
+    victim->last_use = c->step_tick;
+    return step_enqueue(TALON_STEP_ARGS);
+  }
+  hit->last_use = c->step_tick;
+  if (!hit->exec) {                // second sighting: capture
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      c->step_graph = 0;           // this stream or driver cannot capture: stop trying
+      return step_enqueue(TALON_STEP_ARGS);
+    }
+    const long long before = c->launches;
+    const talon_status r = step_enqueue(TALON_STEP_ARGS);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(st, &graph);
+    cudaGraphExec_t exec = nullptr;
+    if (r == TALON_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+      hit->exec = exec;
+      hit->launches = c->launches - before;
+      hit->layers_run = c->layers_run;
+      c->launches = before;        // nothing has run yet: the replay below counts
+    } else {
+      cudaGetLastError();
+      c->launches = before;
+      hit->used = false;           // do not try these arguments again until they are seen anew
+      if (graph) cudaGraphDestroy(graph);
+      if (r != TALON_OK) return r;
+      return step_enqueue(TALON_STEP_ARGS);
+    }
+    cudaGraphDestroy(graph);
+  }
+  if (cudaGraphLaunch(hit->exec, st) != cudaSuccess) return TALON_ERR_CUDA;
+  c->B = B;
+  c->layers_run = hit->layers_run;
+  c->launches += hit->launches;
+  return TALON_OK;
+#undef TALON_STEP_ARGS
 }
 
 talon_status talon_step_host(talon_ctx *c, int32_t B, const int32_t *root_tok, const int32_t *prefix_len,

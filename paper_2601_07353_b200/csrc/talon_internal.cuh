@@ -81,6 +81,20 @@ __host__ __device__ inline LayerGeom make_geom(int total_rows, int vocab, int ta
 
 }  // namespace talon
 
+namespace talon {
+// A whole step captured as a CUDA graph, keyed by every argument of the call that made it.
+constexpr int STEP_GRAPH_SLOTS = 64;
+constexpr int STEP_GRAPH_WORDS = 36;
+struct StepGraph {
+  unsigned long long args[STEP_GRAPH_WORDS];
+  cudaGraphExec_t exec;      // null: arguments seen once, nothing captured yet
+  long long launches;        // kernels one replay launches
+  int layers_run;            // host-side depth counter after the step
+  unsigned long long last_use;
+  bool used;
+};
+}  // namespace talon
+
 // The context: parameters, host-side counters, and the device workspace.
 struct talon_ctx {
   talon_params p;
@@ -125,6 +139,10 @@ struct talon_ctx {
   int ev_cap, ev_used;
   unsigned ev_mask;                  // kernel families that are timed
   int ev_paused;                     // 1: launches are not bracketed for now
+  // talon_step replays (see talon_step)
+  int step_graph;                    // 0: never capture
+  unsigned long long step_tick;
+  talon::StepGraph *graphs;          // [STEP_GRAPH_SLOTS], allocated on first use
 };
 
 namespace talon {

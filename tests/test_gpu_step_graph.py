@@ -1,0 +1,75 @@
+"""talon_step replays a captured graph from the second call with the same arguments: the replays
+must give what the plain launch sequence gives, read their inputs afresh, and count their launches."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_07353_b200 import synth
+from tests import test_gpu_parity as GP
+
+pytestmark = pytest.mark.gpu
+
+
+def _snapshot(wl):
+    tr = wl.tree
+    return [x.clone() for x in (tr.n_nodes, tr.token, tr.parent, tr.depth, tr.position, tr.layer_off, tr.score, tr.mask,
+                                wl.out, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok)]
+
+
+def test_replayed_steps_equal_plain_steps_and_read_fresh_inputs():
+    from paper_2601_07353_b200 import talon, workload
+    cfg = synth.CONFIGS["tiny"].scaled(batch=3, prefix_min=50, prefix_max=400)
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, GP.SEED)
+    workload.run_step(t, wl)                        # entry by entry: the reference result
+    torch.cuda.synchronize()
+    want = _snapshot(wl)
+    per_step = None
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for call in range(5):                       # 1: plain, 2: capture + replay, 3..: replay
+            for x in (wl.tree.token, wl.out, wl.accept_len, wl.bonus_tok):
+                x.zero_()
+            before = t.launch_count()
+            workload.run_step_fused(t, wl)
+            side.synchronize()
+            assert t.poll_status() == talon.OK
+            n = t.launch_count() - before
+            per_step = n if per_step is None else per_step
+            assert n == per_step and n > 0          # replays count the kernels they launch
+            assert t.layers_run() == cfg.max_depth
+            for a, b in zip(want, _snapshot(wl)):
+                assert torch.equal(a, b), f"call {call}"
+        # same pointers, new contents: a replay must pick them up
+        wl.root_tok[0] = (int(wl.root_tok[0]) + 1) % cfg.vocab
+        workload.run_step_fused(t, wl)
+        side.synchronize()
+        assert int(wl.tree.token[0, 0]) == int(wl.root_tok[0])
+    GP.check_verify(cfg, wl, [1, 2])                # untouched sequences still match the oracle
+    t.close()
+
+
+def test_timed_and_default_stream_steps_take_the_plain_path():
+    from paper_2601_07353_b200 import talon, workload
+    cfg = synth.CONFIGS["tiny"]
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, GP.SEED)
+    for _ in range(3):                              # legacy default stream: never captured
+        workload.run_step_fused(t, wl)
+    torch.cuda.synchronize()
+    assert t.poll_status() == talon.OK
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            workload.run_step_fused(t, wl)
+        t.timing_enable(64)
+        workload.run_step_fused(t, wl)              # bracketed by events: launched one by one
+        kt = t.timing_read()
+        assert kt["expand_rows"][1] == cfg.max_depth and kt["tree_attention"][1] == 1
+        t.timing_enable(0)
+        workload.run_step_fused(t, wl)
+        side.synchronize()
+    assert t.poll_status() == talon.OK
+    GP.check_expansion(cfg, wl, [0])
+    GP.check_verify(cfg, wl, [0])
+    t.close()
