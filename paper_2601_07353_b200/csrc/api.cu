@@ -110,14 +110,13 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
   c->key_stride = (k + 3) & ~3;
   c->log_mu = std::log(p->mu);
   {
-    // Programmatic dependent launch is off unless TALON_PDL=1: measured on B200 it gains about 2 %
-    // at batch 1 and loses about 10 % at batch 16, where the early-scheduled CTAs of the next
-    // kernel take SM slots from the running one.
+    // Programmatic dependent launch: measured on B200 it gains about 3 % at batch 1 and loses
+    // 3-10 % at batch 16, so by default it is used for small batches only (TALON_PDL=1 / 0 forces it).
     const char *mt = std::getenv("TALON_ATTN_MIN_TILES");
     c->attn_min_tiles = mt ? std::atoi(mt) : 4;
     if (c->attn_min_tiles < 1) c->attn_min_tiles = 1;
     const char *e = std::getenv("TALON_PDL");
-    c->pdl = (e && e[0] == '1') ? 1 : 0;
+    c->pdl = !e ? -1 : (e[0] == '1' ? 1 : 0);
     const char *g = std::getenv("TALON_STEP_GRAPH");
     c->step_graph = (g && g[0] == '0') ? 0 : 1;
   }

@@ -123,7 +123,7 @@ struct talon_ctx {
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
   int attn_min_tiles;                // split-KV: key tiles a CTA should at least own
-  int pdl;                           // 1: kernels are launched with programmatic stream serialization
+  int pdl;                           // programmatic stream serialization: 1 on, 0 off, -1 on for small batches
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
   int32_t *d_target_tok;             // [batch_max * N]
@@ -156,7 +156,11 @@ __device__ __forceinline__ void pdl_enter() {
 }
 
 // Launches `kernel` so that it may be scheduled while its predecessor in the stream drains
-// (the kernel itself waits in pdl_enter()); a plain launch when ctx->pdl is off.
+// (the kernel itself waits in pdl_enter()); a plain launch when ctx->pdl is off.  In automatic mode
+// (-1) it is used for batches of at most PDL_AUTO_BATCH sequences: there the grids are small and the
+// overlapped launch latency is a gain, while at larger batches the early-scheduled CTAs of the next
+// kernel take SM slots from the running one.
+constexpr int PDL_AUTO_BATCH = 4;
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                                  cudaStream_t st, Args &&...args) {
@@ -169,7 +173,7 @@ inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), d
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = c->pdl ? 1 : 0;
+  cfg.numAttrs = (c->pdl == 1 || (c->pdl < 0 && c->B <= PDL_AUTO_BATCH)) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
