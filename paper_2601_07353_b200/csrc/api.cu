@@ -443,11 +443,12 @@ talon_status talon_step(talon_ctx *c, const talon_tree *t, int32_t B, const int3
       hit->layers_run = c->layers_run;
       c->launches = before;        // nothing has run yet: the replay below counts
     } else {
+      // nothing ran: clean up and do the step the plain way, which also reports a bad argument
       cudaGetLastError();
       c->launches = before;
-      hit->used = false;           // do not try these arguments again until they are seen anew
+      hit->used = false;
       if (graph) cudaGraphDestroy(graph);
-      if (r != TALON_OK) return r;
+      if (r == TALON_OK) c->step_graph = 0;      // the capture itself failed: stop trying
       return step_enqueue(TALON_STEP_ARGS);
     }
     cudaGraphDestroy(graph);
