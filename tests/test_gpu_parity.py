@@ -195,3 +195,19 @@ def test_repeatable_bits():
         for a, b in zip(snaps[0], s):
             assert torch.equal(a, b)
     t.close()
+
+
+def test_more_than_32_sequences():
+    """Above 32 sequences the frontier geometry goes through shared memory instead of registers."""
+    cfg = synth.CONFIGS["tiny"].scaled(vocab=4096, batch=40, prefix_min=3, prefix_max=200)
+    run_config(cfg, heads=[0, 17])
+
+
+@pytest.mark.parametrize("k,budget", [(16, 64), (32, 100), (12, 128)])
+def test_wide_candidate_lists_on_the_fused_kernel(k, budget):
+    """Per-parent caps up to 32 stay on the fused kernel (different lane-group sizes for the bound)."""
+    cfg = synth.CONFIGS["tiny"].scaled(vocab=8192, batch=3, topk=k, budget=budget, max_depth=10, prefix_min=20,
+                                      prefix_max=90)
+    run_config(cfg, heads=[3])
+    cfg = synth.CONFIGS["llama8b"].scaled(batch=2, topk=k, budget=budget, prefix_min=64, prefix_max=64)
+    run_config(cfg, heads=[3])

@@ -154,3 +154,8 @@ def test_one_hot_targets_give_the_greedy_result():
     assert torch.equal(o["alen"], wl.accept_len) and torch.equal(o["nodes"], wl.accept_nodes)
     assert torch.equal(o["tok"], wl.bonus_tok)
     t.close()
+
+
+def test_more_than_32_sequences():
+    cfg = synth.CONFIGS["tiny"].scaled(vocab=4096, batch=40, prefix_min=3, prefix_max=200)
+    sample_and_check(cfg, temperatures=(1.0, 0.3), draws=1)
