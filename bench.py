@@ -472,7 +472,7 @@ def run_talon(args, cfg):
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
                 "traffic": None if ratio is None else ratio * dom_bytes_total * timed_frac / dom_n,
                 "traffic_source": None if ratio is None else "ncu capture of an earlier run, same kernel source: DRAM bytes per algorithmic byte x this run's bytes per launch",
-                "launches_timed": int(dom_n), "timed_steps": f"every {TIMED_EVERY}th step of the timed region", "avg_launch_us": dom_ms / dom_n * 1e3,
+                "launches_timed": int(dom_n), "timed_steps": f"1 step in {TIMED_EVERY} of the timed region", "avg_launch_us": dom_ms / dom_n * 1e3,
                 "algorithmic_bytes_per_launch": dom_bytes_total * timed_frac / dom_n}
         if dominant == "tree_attention" and intensity > ridge:
             tf = dom_flops_total * timed_frac / (dom_ms * 1e-3) / 1e12
