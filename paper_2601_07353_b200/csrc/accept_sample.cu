@@ -7,9 +7,11 @@
 //   accept_sample_kernel        : one CTA per sequence.  Chunk statistics -> log-sum-exp per node;
 //                                 warp 0 walks from the root and tries the children of the current
 //                                 node one after the other (child with token w accepted when
-//                                 u * unclaimed mass < p(w), else w is struck); the whole CTA then
-//                                 draws the correction token from what is left of the posterior at
-//                                 the last node by inverse CDF in token order (step 3).
+//                                 u * unclaimed mass < p(w), else w is struck); the CTA then draws
+//                                 the correction token from what is left of the posterior at the
+//                                 last node by inverse CDF in token order (step 3): the chunk
+//                                 statistics of that row say which chunk holds the target mass, so
+//                                 only that chunk of the row is read again.
 //
 // The uniforms are inputs: one per node (consumed if the node is tried) and one per sequence.
 #include <math_constants.h>
@@ -122,7 +124,7 @@ struct SampleArgs {
   int B, N, V, max_depth;
   const float *logits;
   int64_t row_stride;
-  int splits;
+  int splits, chunk_len;
   const float2 *part;
   float scale;              // log2(e) / T
   double inv_t;             // 1 / T
@@ -145,8 +147,9 @@ accept_sample_kernel(SampleArgs a) {
   __shared__ int s_rej[SAMP_MAX_NODES];           // tokens struck at the last node
   __shared__ double s_gsum[SAMP_MAX_GROUPS];        // weight of each group of 128 tokens
   __shared__ double s_wtot[SAMP_WARPS];
-  __shared__ int s_cur, s_nrej, s_bad, s_pick;
-  __shared__ double s_resid;
+  __shared__ double s_rejw[SAMP_MAX_NODES];         // their weights
+  __shared__ int s_cur, s_nrej, s_bad, s_pick, s_chunk;
+  __shared__ double s_resid, s_cw;
 
   pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -157,20 +160,23 @@ accept_sample_kernel(SampleArgs a) {
   if (tid == 0) { s_bad = 0; s_pick = -1; }
   __syncthreads();
 
-  // ---- step (1): the normaliser of every node's posterior from the chunk statistics ----
-  for (int i = tid; i < n; i += SAMP_THREADS) {
-    const float2 *pp = a.part + (nb + i) * a.splits;
-    float mx = -CUDART_INF_F;
-    for (int c = 0; c < a.splits; ++c) mx = fmaxf(mx, pp[c].x);
+  // ---- step (1): the normaliser of every node's posterior from the chunk statistics:
+  // one warp per node, one lane per chunk (at most 32 chunks) ----
+  for (int i = warp; i < n; i += SAMP_WARPS) {
+    const float2 ms = lane < a.splits ? a.part[(nb + i) * a.splits + lane] : make_float2(-CUDART_INF_F, 0.f);
+    float mx = ms.x;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
     double t = 0.0;
-    for (int c = 0; c < a.splits; ++c) {
-      const float2 ms = pp[c];
-      if (ms.y != ms.y) t += (double)ms.y;
-      else if (ms.x > -CUDART_INF_F) t += (double)ms.y * (double)exp2f((ms.x - mx) * a.scale);
+    if (ms.y != ms.y) t = (double)ms.y;
+    else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * a.scale);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
+    if (lane == 0) {
+      if (!(t > 0.0) || !(t < CUDART_INF) || !(mx < CUDART_INF_F) || !(mx > -CUDART_INF_F)) s_bad = 1;
+      s_max[i] = mx;
+      s_logt[i] = log(t);
     }
-    if (!(t > 0.0) || !(t < CUDART_INF) || !(mx < CUDART_INF_F) || !(mx > -CUDART_INF_F)) s_bad = 1;
-    s_max[i] = mx;
-    s_logt[i] = log(t);
   }
   __syncthreads();
   if (s_bad) {                  // a posterior that does not exist: nothing is accepted, no token
@@ -239,20 +245,70 @@ accept_sample_kernel(SampleArgs a) {
   const int cur = s_cur, nrej = s_nrej;
   const float *rowp = a.logits + (int64_t)(nb + cur) * a.row_stride;
   const float rmax = s_max[cur];
-  const int groups = (a.V + SAMP_GROUP - 1) / SAMP_GROUP;
+  // (a) which chunk of the row holds the target mass: the chunk statistics already say how much
+  // weight each chunk carries; the struck tokens are taken out of their chunks first
+  if (warp == 0) {
+    const float2 ms = lane < a.splits ? a.part[(nb + cur) * a.splits + lane] : make_float2(-CUDART_INF_F, 0.f);
+    double wc = (ms.x > -CUDART_INF_F) ? (double)ms.y * (double)exp2f((ms.x - rmax) * a.scale) : 0.0;
+    for (int r0 = 0; r0 < nrej; r0 += 32) {
+      const int r = r0 + lane;
+      const int w = r < nrej ? s_rej[r] : 0;
+      const double wt = r < nrej ? weight(rowp[w], rmax, a.scale) : 0.0;
+      if (r < nrej) s_rejw[r] = wt;
+      for (int j = 0; j < min(32, nrej - r0); ++j) {          // in storage order, one after the other
+        const int wj = __shfl_sync(FULL, w, j);
+        const double tj = __shfl_sync(FULL, wt, j);
+        if (lane == wj / a.chunk_len) wc -= tj;
+      }
+    }
+    wc = fmax(wc, 0.0);
+    double inc = wc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double t = __shfl_up_sync(FULL, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const double total = __shfl_sync(FULL, inc, 31);
+    const double target = a.u_sample[b] * total;
+    const double excl = inc - wc;
+    const unsigned here = __ballot_sync(FULL, wc > 0.0 && excl <= target && target < inc);
+    const unsigned any = __ballot_sync(FULL, wc > 0.0);
+    int c;
+    double resid, cw;
+    if (here) {
+      c = __ffs(here) - 1;
+      resid = target - __shfl_sync(FULL, excl, c);
+    } else {                       // rounding put the target at or past the total: the last chunk with weight
+      c = any ? 31 - __clz(any) : -1;
+      resid = CUDART_INF;
+    }
+    cw = c >= 0 ? __shfl_sync(FULL, wc, c) : 0.0;
+    if (lane == 0) { s_chunk = c; s_resid = resid; s_cw = cw; }
+  }
+  __syncthreads();
+  const int chunk = s_chunk;
+  const double chunk_resid = s_resid, chunk_weight = s_cw;      // read before anybody reuses the slots
+  if (chunk < 0) {                 // no weight at all (cannot happen with a finite row)
+    if (tid == 0) a.out_tok[b] = -1;
+    return;
+  }
+  // (b) weights of the chosen chunk's groups of 128 tokens: one 128-bit load per lane, all of a
+  // warp's loads requested before any is used
+  const int c_lo = chunk * a.chunk_len, c_hi = min(a.V, c_lo + a.chunk_len);
+  const int groups = (c_hi - c_lo + SAMP_GROUP - 1) / SAMP_GROUP;
   for (int g0 = warp; g0 < groups; g0 += 4 * SAMP_WARPS) {
     float4 x[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const int g = g0 + r * SAMP_WARPS;
-      const int idx = g * SAMP_GROUP + lane * 4;
+      const int idx = c_lo + g * SAMP_GROUP + lane * 4;
       x[r] = make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
       if (g < groups) {
-        if (idx + 4 <= a.V) x[r] = *reinterpret_cast<const float4 *>(rowp + idx);
+        if (idx + 4 <= c_hi) x[r] = *reinterpret_cast<const float4 *>(rowp + idx);
         else {
-          if (idx < a.V) x[r].x = rowp[idx];
-          if (idx + 1 < a.V) x[r].y = rowp[idx + 1];
-          if (idx + 2 < a.V) x[r].z = rowp[idx + 2];
+          if (idx < c_hi) x[r].x = rowp[idx];
+          if (idx + 1 < c_hi) x[r].y = rowp[idx + 1];
+          if (idx + 2 < c_hi) x[r].z = rowp[idx + 2];
         }
       }
     }
@@ -267,10 +323,10 @@ accept_sample_kernel(SampleArgs a) {
     }
   }
   __syncthreads();
-  if (tid == 0)                                   // strike the rejected tokens (a handful), in order
+  if (tid == 0)                                   // strike the rejected tokens of this chunk, in order
     for (int r = 0; r < nrej; ++r) {
       const int w = s_rej[r];
-      s_gsum[w / SAMP_GROUP] -= weight(rowp[w], rmax, a.scale);
+      if (w >= c_lo && w < c_hi) s_gsum[(w - c_lo) / SAMP_GROUP] -= s_rejw[r];
     }
   __syncthreads();
   // inclusive scan of the group weights in token order: thread t owns groups 2t, 2t+1
@@ -299,8 +355,10 @@ accept_sample_kernel(SampleArgs a) {
     s_wtot[lane] = w;                             // inclusive over warps
   }
   __syncthreads();
+  // the target inside the chunk, on the scale of the weights just recomputed (the chunk statistic
+  // and the recomputed total agree to rounding; the ratio keeps the relative position)
   const double total = s_wtot[SAMP_WARPS - 1];
-  const double target = a.u_sample[b] * total;
+  const double target = chunk_resid < CUDART_INF ? chunk_resid * (total / chunk_weight) : CUDART_INF;
   double excl = (warp ? s_wtot[warp - 1] : 0.0) + inc - local;
 #pragma unroll
   for (int r = 0; r < SAMP_GROUPS_PER_THREAD; ++r) {
@@ -327,11 +385,11 @@ accept_sample_kernel(SampleArgs a) {
     return;
   }
   // inside the group: 4 tokens per lane in token order
-  const int idx = g * SAMP_GROUP + lane * 4;
+  const int idx = c_lo + g * SAMP_GROUP + lane * 4;
   double wv[4];
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    wv[e] = idx + e < a.V ? weight(rowp[idx + e], rmax, a.scale) : 0.0;
+    wv[e] = idx + e < c_hi ? weight(rowp[idx + e], rmax, a.scale) : 0.0;
     for (int r = 0; r < nrej; ++r)
       if (s_rej[r] == idx + e) wv[e] = 0.0;
   }
@@ -390,7 +448,7 @@ talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float
   wa.t = *t; wa.lo_stride = c->p.max_depth + 2;
   wa.B = c->B; wa.N = c->p.budget; wa.V = c->p.vocab; wa.max_depth = c->p.max_depth;
   wa.logits = target_logits; wa.row_stride = row_stride;
-  wa.splits = g.splits; wa.part = c->d_samp_ms;
+  wa.splits = g.splits; wa.chunk_len = g.chunk_len; wa.part = c->d_samp_ms;
   wa.scale = sa.scale; wa.inv_t = 1.0 / temperature;
   wa.u_accept = u_accept; wa.u_sample = u_sample;
   wa.accept_len = accept_len; wa.accept_nodes = accept_nodes; wa.out_tok = out_tok;
