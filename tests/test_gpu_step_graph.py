@@ -73,3 +73,23 @@ def test_timed_and_default_stream_steps_take_the_plain_path():
     GP.check_expansion(cfg, wl, [0])
     GP.check_verify(cfg, wl, [0])
     t.close()
+
+
+@pytest.mark.parametrize("name,seqs,heads", [("llama8b", None, None), ("llama8b_batched", [0, 9, 15], [0, 31])])
+def test_full_size_replayed_step_matches_the_oracle(name, seqs, heads):
+    """The launch configuration the benchmark times (talon_step on its own stream, replaying its
+    captured graph) against the oracle at full size."""
+    from paper_2601_07353_b200 import talon, workload
+    cfg = synth.CONFIGS[name]
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, GP.SEED)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(4):
+            workload.run_step_fused(t, wl)
+        side.synchronize()
+    assert t.poll_status() == talon.OK
+    check = list(range(wl.B)) if seqs is None else seqs
+    GP.check_expansion(cfg, wl, check)
+    GP.check_verify(cfg, wl, check, heads)
+    t.close()
