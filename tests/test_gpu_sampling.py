@@ -159,3 +159,37 @@ def test_one_hot_targets_give_the_greedy_result():
 def test_more_than_32_sequences():
     cfg = synth.CONFIGS["tiny"].scaled(vocab=4096, batch=40, prefix_min=3, prefix_max=200)
     sample_and_check(cfg, temperatures=(1.0, 0.3), draws=1)
+
+
+def test_many_struck_children_in_the_full_pool_mode():
+    """With the paper's whole-vocabulary pool a parent can hold dozens of children: walk to the node
+    with the most children (uniform 0 along the way), reject them all there (uniform just below 1) and
+    draw from what is left."""
+    talon, workload = _mods()
+    cfg = synth.CONFIGS["llama8b"].scaled(vocab=2048, batch=4, prefix_min=10, prefix_max=90, budget=100, mu=1e-4,
+                                          spike="none")
+    t = workload.make_talon(cfg, cand_topk=0)
+    wl = workload.build_workload(cfg, t, SEED)
+    N, dev, B = cfg.budget, wl.target.device, wl.B
+    trees = [PU.oracle_tree_from_arrays(PU.tree_to_host(wl.tree, bi), N, cfg.max_depth) for bi in range(B)]
+    ua = np.full((B, N), 1.0 - 2.0 ** -53)
+    most = []
+    for bi, tr in enumerate(trees):
+        kids = [len(O.children_of(tr, v)) for v in range(tr.n_nodes)]
+        end = int(np.argmax(kids))
+        most.append(kids[end])
+        v = end
+        while v > 0:                      # accept everything on the way down to `end`
+            ua[bi, v] = 0.0
+            v = int(tr.parent[v])
+    assert max(most) > 32, most
+    alen = torch.zeros(B, dtype=torch.int32, device=dev)
+    nodes = torch.zeros(B, cfg.max_depth + 1, dtype=torch.int32, device=dev)
+    tok = torch.zeros(B, dtype=torch.int32, device=dev)
+    us = np.array([0.1, 0.5, 0.9, 0.999])
+    t.accept_sample(wl.tree, wl.target, 1.0, torch.from_numpy(ua).to(dev), torch.from_numpy(us).to(dev), alen, nodes, tok)
+    assert t.poll_status() == talon.OK
+    for bi in range(B):
+        PU.follow_sampling(trees[bi], wl.target[bi].cpu().numpy(), ua[bi], float(us[bi]), 1.0, int(alen[bi]),
+                           nodes[bi].cpu().numpy(), int(tok[bi]), f"full pool [{bi}]")
+    t.close()
