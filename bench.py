@@ -516,6 +516,59 @@ def run_talon(args, cfg):
     return 0
 
 
+# --------------------------------------------------------------------------------------------
+# the paper's own on-path experiment: single-layer tree-expansion latency on Zipf rows
+# --------------------------------------------------------------------------------------------
+def run_zipf_micro(args):
+    """Latency of one expansion layer (the K children of the root as frontier, batch 1) on rows with
+    P(rank r) ~ r^-alpha, for the paper's vocabularies and exponents: 20 warm-up runs, mean of 100,
+    as in the appendix's tree-construction micro-benchmark.  Extra mode; prints its own JSON line."""
+    import torch
+    from paper_2601_07353_b200 import roofline, synth, talon
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = roofline.load_peaks(ROOT)
+    N, K, D = 60, 10, 8
+    results = []
+    for V in (32000, 128256, 151936):
+        t = talon.Talon(batch_max=1, vocab=V, budget=N, root_topk=K, cand_topk=K, max_depth=D, mu=0.03,
+                        n_q_heads=32, n_kv_heads=8, head_dim=128, device=0)
+        tree = t.alloc_tree(1)
+        root = torch.zeros(1, dtype=torch.int32, device=dev)
+        plen = torch.zeros(1, dtype=torch.int32, device=dev)
+        draft = torch.zeros(1, N, V, dtype=torch.float32, device=dev)
+        for alpha in (0.7, 1.35, 5.0):
+            for i in range(K + 1):                    # the root's row and the rows of its K children
+                draft[0, i] = synth.zipf_logits_row(V, alpha, args.seed, i, device=dev)
+            e0 = [torch.cuda.Event(enable_timing=True) for _ in range(120)]
+            e1 = [torch.cuda.Event(enable_timing=True) for _ in range(120)]
+            for it in range(120):
+                t.reset(tree, root, plen)
+                t.expand_layer(tree, draft)           # root layer (Top-K): untimed
+                e0[it].record()
+                t.expand_layer(tree, draft)           # the timed layer: K frontier rows, gate, truncation
+                e1[it].record()
+            torch.cuda.synchronize()
+            assert t.poll_status() == talon.OK
+            lo = tree.layer_off[0].cpu().tolist()
+            rows = lo[2] - lo[1]
+            us = [a.elapsed_time(b) * 1e3 for a, b in zip(e0[20:], e1[20:])]
+            mean = sum(us) / len(us)
+            results.append({"vocab": V, "alpha": alpha, "frontier_rows": rows, "nodes_added": lo[3] - lo[2],
+                            "us_mean": mean, "us_min": min(us),
+                            "algorithmic_gbs": 4.0 * V * rows / (mean * 1e-6) / 1e9})
+        t.close()
+    print(json.dumps({"metric": "single-layer tree-expansion latency (Zipf rows, warm caches)", "unit": "us",
+                      "higher_is_better": False, "n_gpus": 1, "data": "synthetic",
+                      "config": {"workload": "batch 1, budget 60, K 10, frontier = the root's children; "
+                                             "20 warm-up runs, mean of 100, events around the launch"},
+                      "peak_hbm_gbs": peaks["hbm_gbs"], "results": results}))
+    return 0
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -530,10 +583,14 @@ def main(argv=None):
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sampling", action="store_true", help="skip the sampling-verification extra")
+    ap.add_argument("--zipf-micro", action="store_true",
+                    help="instead of the step benchmark: single-layer expansion latency on Zipf rows")
     args = ap.parse_args(argv)
     from paper_2601_07353_b200 import synth
     if args.seed is None:
         args.seed = synth.DEFAULT_SEED
+    if args.zipf_micro:
+        return run_zipf_micro(args)
     cfg = synth.CONFIGS[args.config]
     if args.impl == "reference":
         args.steps = 10 if args.steps is None else args.steps

@@ -211,3 +211,45 @@ def test_wide_candidate_lists_on_the_fused_kernel(k, budget):
     run_config(cfg, heads=[3])
     cfg = synth.CONFIGS["llama8b"].scaled(batch=2, topk=k, budget=budget, prefix_min=64, prefix_max=64)
     run_config(cfg, heads=[3])
+
+
+@pytest.mark.parametrize("alpha", [0.7, 1.35, 5.0])
+def test_zipf_rows_of_the_papers_micro_benchmark(alpha):
+    """Expansion on the appendix's Zipf rows (P(rank r) ~ r^-alpha): the same tree as the oracle's.
+    Each row is generated once on the host and handed to both sides."""
+    talon, workload = _mods()
+    V, N, K, D = 32000, 60, 10, 8
+    t = talon.Talon(batch_max=1, vocab=V, budget=N, root_topk=K, cand_topk=K, max_depth=D, mu=0.03, n_q_heads=32,
+                    n_kv_heads=8, head_dim=128)
+    rows = {}
+
+    def row(path):                                    # a node's row depends on its token path only
+        key = tuple(path)
+        if key not in rows:
+            rows[key] = synth.zipf_logits_row(V, alpha, 5, len(rows))
+        return rows[key]
+
+    p = O.Params(N, K, K, 0.03, D)
+    want = O.expand(7, row, p)
+    tree = t.alloc_tree(1)
+    dev = tree.token.device
+    draft = torch.zeros(1, N, V, dtype=torch.float32, device=dev)
+    t.reset(tree, torch.tensor([7], dtype=torch.int32, device=dev), torch.zeros(1, dtype=torch.int32, device=dev))
+    for d in range(D):
+        n = int(tree.n_nodes[0])
+        tok, par = tree.token[0].cpu().numpy(), tree.parent[0].cpu().numpy()
+        paths = workload.node_paths(tok, par, n)
+        for i in range(n):
+            draft[0, i] = torch.from_numpy(row(paths[i])).to(dev)
+        t.expand_layer(tree, draft)
+    t.build_tree(tree)
+    assert t.poll_status() == talon.OK
+    g = PU.tree_to_host(tree, 0)
+    # every row is a permutation of the same values, so path scores of different parents tie exactly
+    # in exact arithmetic: the comparison goes through the tolerated-tie rule
+    followed, tolerated = PU.follow_tree(None, p, 7, row, g["token"], g["parent"], g["n_nodes"], g["layer_off"],
+                                         f"zipf alpha {alpha}")
+    PU.compare_tree_arrays(O.finalize(followed, 0), g, f"zipf alpha {alpha}")
+    assert want.n_nodes == g["n_nodes"]
+    print(f"zipf alpha {alpha}: n_nodes {g['n_nodes']}, tolerated ties {tolerated}")
+    t.close()
