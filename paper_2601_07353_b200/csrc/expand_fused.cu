@@ -341,8 +341,10 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int l
   // One warp per row, one lane per chunk (S <= 32). ----
   const int stage_words = 32 * k + FX_SURV;
   // Many rows means few chunks per row (their product is bounded by the grid): then all rows
-  // are merged at once, one thread per key, instead of a row at a time per warp.
-  const bool flat = S > 1 && S <= 8 && F > EXP_WARPS && F * S * k <= EXP_WARPS * stage_words;
+  // are merged at once, one thread per key, instead of a row at a time per warp.  Up to two
+  // rounds of the warp-per-row merge measured faster than the flat one (10 rows x 8 chunks:
+  // 4 us per layer), hence the bound on F.
+  const bool flat = S > 1 && S <= 8 && F > 2 * EXP_WARPS && F * S * k <= EXP_WARPS * stage_words;
   if (flat) {
     const size_t item0 = (size_t)row0 * S;
     u64 *st = sm.stage;                           // st[(j * S + c) * k + i]
