@@ -483,6 +483,7 @@ def run_talon(args, cfg):
         if k in kernels and kernels[k]["ms_per_step"] > 0:
             kernels[k]["algorithmic_gbs"] = per_step[k] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
             kernels[k]["frac_of_hbm_peak"] = kernels[k]["algorithmic_gbs"] / peaks["hbm_gbs"]
+            kernels[k]["frac_of_nominal_8tbs"] = kernels[k]["algorithmic_gbs"] / 8000.0
     if "tree_attention" in kernels:
         kernels["tree_attention"]["tflops"] = att_flops_step / (kernels["tree_attention"]["ms_per_step"] * 1e-3) / 1e12
 
