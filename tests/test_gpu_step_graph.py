@@ -93,3 +93,29 @@ def test_full_size_replayed_step_matches_the_oracle(name, seqs, heads):
     GP.check_expansion(cfg, wl, check)
     GP.check_verify(cfg, wl, check, heads)
     t.close()
+
+
+def test_more_argument_sets_than_graph_slots():
+    """The library keeps 64 captured steps; with 70 argument sets in rotation the least recently used
+    ones are dropped and re-captured, and every step still gives the same result."""
+    from paper_2601_07353_b200 import talon, workload
+    cfg = synth.CONFIGS["tiny"].scaled(vocab=4096, batch=2, prefix_min=30, prefix_max=60)
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, GP.SEED)
+    workload.run_step(t, wl)
+    torch.cuda.synchronize()
+    want = wl.out.clone()
+    want_tok = wl.tree.token.clone()
+    outs = [torch.zeros_like(wl.out) for _ in range(70)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for rnd in range(3):
+            for o in outs:
+                wl.out = o                      # a different output pointer is a different argument set
+                workload.run_step_fused(t, wl)
+        side.synchronize()
+    assert t.poll_status() == talon.OK
+    for o in outs:
+        assert torch.equal(o, want)
+    assert torch.equal(wl.tree.token, want_tok)
+    t.close()
