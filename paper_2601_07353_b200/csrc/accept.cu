@@ -40,19 +40,30 @@ target_argmax_kernel(ArgmaxArgs a) {
     float bestv = -CUDART_INF_F;
     uint32_t besti = 0xFFFFFFFFu;
     bool bad = false;
-    for (int base = start; base < end; base += EXP_TILE) {
-      float v[EXP_UNROLL][EXP_VEC];
+    // the next tile is requested before the current one is worked on: a chunk of a few tiles is a
+    // chain of DRAM round trips otherwise
+    float nx[EXP_UNROLL][EXP_VEC];
+    auto load = [&](int base) {
 #pragma unroll
       for (int u = 0; u < EXP_UNROLL; ++u) {
         const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
         if (idx + EXP_VEC <= end) {
           const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
-          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+          nx[u][0] = x.x; nx[u][1] = x.y; nx[u][2] = x.z; nx[u][3] = x.w;
         } else {
 #pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
+          for (int e = 0; e < EXP_VEC; ++e) nx[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
         }
       }
+    };
+    load(start);
+    for (int base = start; base < end; base += EXP_TILE) {
+      float v[EXP_UNROLL][EXP_VEC];
+#pragma unroll
+      for (int u = 0; u < EXP_UNROLL; ++u)
+#pragma unroll
+        for (int e = 0; e < EXP_VEC; ++e) v[u][e] = nx[u][e];
+      if (base + EXP_TILE < end) load(base + EXP_TILE);
       // the tile's maximum first (one max per element); only a tile that raises the thread's
       // maximum, or the thread's first tile, is searched for where that maximum sits
       float bm = -CUDART_INF_F;
