@@ -154,7 +154,8 @@ talon_status talon_tree_attention(talon_ctx *ctx, const talon_tree *tree, const 
 
 /* Greedy verification (Appendix B steps 1-2 at temperature 0): t_i = argmax of the target
  * logits after node i (lowest id among equal maxima), then from the root follow the child
- * whose token equals t_cur until none does.
+ * whose token equals t_cur until none does.  Call after talon_build_tree (the walk reads the closed
+ * layer offsets).
  * target_logits device fp32, row of node i of sequence b at (b*N + i) * row_stride; 16-byte aligned rows
  * target_tok    device [B, N] or null: receives t_i (-1 for unused slots)
  * accept_len    device [B]: number of accepted draft tokens (root not counted)
@@ -171,7 +172,8 @@ talon_status talon_accept(talon_ctx *ctx, const talon_tree *tree, const float *t
  * first), the children of that node are tried in storage order: child c with token w is
  * accepted when u_accept[c] * (mass not yet struck) < p(w), otherwise w is struck from p.  The
  * first accepted child becomes the current node; when none is accepted the correction token is
- * drawn from what is left of p by inverse CDF in token order with u_sample.
+ * drawn from what is left of p by inverse CDF in token order with u_sample.  Call after
+ * talon_build_tree (the walk reads the closed layer offsets).
  * target_logits device fp32, row of node i of sequence b at (b*N + i) * row_stride; 16-byte aligned rows
  * temperature   host value, > 0
  * u_accept      device [B, N] fp64 uniforms in [0, 1): node c consumes u_accept[b, c] if it is tried
@@ -193,8 +195,8 @@ talon_status talon_accept_sample(talon_ctx *ctx, const talon_tree *tree, const f
  * prefix_len[b] + accept_len[b] of the sequence's block, prefix_len[b] grows by accept_len[b] + 1,
  * root_tok[b] becomes next_tok[b] (talon_accept's bonus_tok or talon_accept_sample's out_tok), and
  * counters[b] advances by (1, draft passes, accept_len[b] + 1): the N_p, N_q and L of Section 5.3,
- * a draft pass being a layer Algorithm 2 expanded for this sequence.  The next step starts with
- * talon_reset(root_tok, prefix_len).
+ * a draft pass being a layer Algorithm 2 expanded for this sequence.  Call after talon_build_tree and
+ * one of the two verification calls.  The next step starts with talon_reset(root_tok, prefix_len).
  * All pointers device memory.  k_tree, v_tree [B, N, Hkv, Dh] bf16; k_prefix, v_prefix, kv_start,
  * kv_tokens, kv_stride_t, kv_stride_h as in talon_tree_attention (written here);
  * kv_limit  [B] int64 or null: first token offset past the block of sequence b (kv_tokens if null)
