@@ -113,7 +113,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     // Programmatic dependent launch: measured on B200 it gains about 3 % at batch 1 and loses
     // 3-10 % at batch 16, so by default it is used for small batches only (TALON_PDL=1 / 0 forces it).
     const char *mt = std::getenv("TALON_ATTN_MIN_TILES");
-    c->attn_min_tiles = mt ? std::atoi(mt) : 4;
+    c->attn_min_tiles = mt ? std::atoi(mt) : 2;
     if (c->attn_min_tiles < 1) c->attn_min_tiles = 1;
     const char *e = std::getenv("TALON_PDL");
     c->pdl = !e ? -1 : (e[0] == '1' ? 1 : 0);
