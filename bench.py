@@ -9,18 +9,24 @@ the N tree tokens against the prefix KV cache, target argmax and the greedy acce
 and target model forwards are not part of the path: their outputs (fp32 logits, bf16 Q/K/V) are
 seeded synthetic tensors, resident in HBM before the timed region starts.
 
+Without ``--config`` the headline is the largest workload that fits one GPU (``longctx``) and the
+other four workloads are measured in the same invocation and reported under ``configs``.
+
 The timed region is K back-to-back ``talon_step`` calls that rotate over enough distinct input sets
 that the bytes touched between two uses of a set exceed the L2 capacity several times over, so
 every step reads its inputs from HBM.  It is bracketed by a barrier and a device synchronisation on
-both sides, timed with CUDA events, and reported as the maximum over ranks.  With more than one
-GPU every rank runs its own replicas (sequences are independent: no data-path collective).
+both sides, timed with CUDA events, and reported as the maximum over ranks.  When K steps take less
+than half a second the region is repeated and the median repeat is reported (``repeats``,
+``spread``), so that clock samples fall inside it.  With more than one GPU every rank runs its own
+replicas (sequences are independent: no data-path collective).
 
-Rank 0 prints one JSON line.  Beside the contract's keys it carries ``roofline`` (the dominant
-kernel's algorithmic bytes over its event-timed launches of the timed region, against the measured
-copy bandwidth), ``cpu_baseline`` (the fp64 CPU oracle timed on a bounded sample), ``e2e`` (the same
-step through ``talon_step_host`` with pinned host buffers), ``graph_replay`` (the step captured in a
-CUDA graph), ``kernels`` (per-kernel time from a separate bracketed pass) and ``tree_shapes``.
-``--impl reference`` times the CPU oracle alone, on host cores.
+Rank 0 prints one JSON line.  Beside the contract's keys it carries ``kernels`` (each kernel family
+timed alone: one event pair around at least 20 back-to-back graph replays of just those launches,
+inputs rotated, so no event bracket sits between two kernels), ``roofline`` (the dominant kernel's
+algorithmic bytes or flops over that duration, against the measured peaks), ``cpu_baseline`` (the
+fp64 CPU oracle on all host cores, one core beside it, with its per-stage split and the count of
+tolerated selection ties), ``e2e`` (the same step through ``talon_step_host`` with pinned host
+buffers), ``tree_shapes`` and ``configs``.  ``--impl reference`` times the CPU oracle alone.
 """
 from __future__ import annotations
 
@@ -44,7 +50,12 @@ METRIC = "draft+verify steps/sec"
 UNIT = "steps/s"
 L2_BYTES = 126 * 1024 * 1024
 ROTATION_FACTOR = 3.0            # bytes between two uses of an input set, in units of L2
-TIMED_EVERY = 32                 # the dominant kernel is event-bracketed on every 32nd timed step
+MIN_REGION_S = 0.5               # a timed region shorter than this is repeated
+KERNEL_REPLAYS = 24              # back-to-back replays per kernel-alone measurement (at least 20)
+HEADLINE = "longctx"
+SUB_CONFIGS = ["tiny", "llama8b", "llama8b_batched", "qwen32b"]
+ORACLE_PREFIX_SAMPLE = 4096      # prefix tokens the oracle's attention is timed on when the prefix is longer
+DTYPE = "f32 logits, f64 path scores, bf16 attention (f32 accumulate)"
 
 
 # --------------------------------------------------------------------------------------------
@@ -97,7 +108,7 @@ class ClockSampler:
     def summary(self, t0: float, t1: float):
         inside = [s for s in self.samples if t0 <= s[0] <= t1]
         window = "timed region"
-        if len(inside) < 3:          # a short timed region sees few samples: take the whole busy span
+        if len(inside) < 3:          # too few samples inside: take the whole busy span and say so
             inside = list(self.samples)
             window = "warm-up to end of run"
         if not inside:
@@ -111,98 +122,138 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # the oracle as a timed CPU baseline (the only place outside tests/ and smoke that runs it)
 # --------------------------------------------------------------------------------------------
-class OracleStep:
-    """One draft-and-verify step of one sequence through the CPU oracle, inputs prepared up front."""
+def oracle_heads(cfg):
+    """Attention heads the oracle is timed on: all of them when that stays within seconds, else
+    three (first, middle, last), scaled to all."""
+    all_heads = cfg.n_q_heads * (min(cfg.prefix_max, ORACLE_PREFIX_SAMPLE) + cfg.budget) <= 32 * 4300
+    return list(range(cfg.n_q_heads)) if all_heads else [0, cfg.n_q_heads // 2, cfg.n_q_heads - 1]
 
-    def __init__(self, cfg, seed: int, seq_id: int, heads):
+
+class OracleStep:
+    """One draft-and-verify step of one sequence through the CPU oracle, inputs prepared up front.
+    A prefix longer than ORACLE_PREFIX_SAMPLE tokens is cut to that length for the attention stage
+    and the stage's time scaled by the key count (attention is linear in it)."""
+
+    def __init__(self, cfg, seed: int, seq_id: int):
         from oracle import talon_oracle as O
         from paper_2601_07353_b200 import synth
-        self.O, self.cfg, self.heads = O, cfg, list(heads)
+        self.O, self.cfg, self.seed, self.seq_id = O, cfg, seed, seq_id
+        self.heads = oracle_heads(cfg)
         self.p = O.Params(cfg.budget, cfg.topk, cfg.topk, cfg.mu, cfg.max_depth)
         self.root = synth.root_token(cfg, seed, seq_id)
         self.L = synth.prefix_len(cfg, seed, seq_id)
+        self.L_used = min(self.L, ORACLE_PREFIX_SAMPLE)
         self.rows = {}
-        gen = lambda path: synth.draft_logits_row(cfg, seed, seq_id, path)
 
         def cached(path):
             key = tuple(path)
             if key not in self.rows:
-                self.rows[key] = gen(path)
+                self.rows[key] = synth.draft_logits_row(cfg, seed, seq_id, path)
             return self.rows[key]
         self.logits_fn = cached
         tree = O.expand(self.root, cached, self.p)        # untimed pass: fills the row cache
+        self.tree = tree
         n, N = tree.n_nodes, cfg.budget
         self.target = np.zeros((N, cfg.vocab), np.float32)
         for i in range(n):
             self.target[i] = synth.target_logits_row(cfg, seed, seq_id, O.path_tokens(tree, i))
-        Hq, Hkv, Dh, g = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.group
-        kvs = sorted({h // g for h in self.heads})
-        q = synth.qkv_block(seed, synth.STREAM_Q, seq_id, N * Hq * Dh).reshape(N, Hq, Dh)
-        kt = synth.qkv_block(seed, synth.STREAM_KT, seq_id, N * Hkv * Dh).reshape(N, Hkv, Dh)
-        vt = synth.qkv_block(seed, synth.STREAM_VT, seq_id, N * Hkv * Dh).reshape(N, Hkv, Dh)
-        kp = np.zeros((self.L, Hkv, Dh), np.float32)
-        vp = np.zeros((self.L, Hkv, Dh), np.float32)
-        step = 4096
-        for t0 in range(0, self.L, step):
-            t1 = min(self.L, t0 + step)
-            cnt, off = (t1 - t0) * Hkv * Dh, t0 * Hkv * Dh
-            kp[t0:t1] = synth.qkv_block(seed, synth.STREAM_K, seq_id, cnt, None, off).reshape(-1, Hkv, Dh)
-            vp[t0:t1] = synth.qkv_block(seed, synth.STREAM_V, seq_id, cnt, None, off).reshape(-1, Hkv, Dh)
-        self.q, self.kt, self.vt, self.kp, self.vp, self.kvs = q, kt, vt, kp, vp, kvs
+        Hq, Hkv, Dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+        self.q = synth.qkv_block(seed, synth.STREAM_Q, seq_id, N * Hq * Dh).reshape(N, Hq, Dh)
+        self.kt = synth.qkv_block(seed, synth.STREAM_KT, seq_id, N * Hkv * Dh).reshape(N, Hkv, Dh)
+        self.vt = synth.qkv_block(seed, synth.STREAM_VT, seq_id, N * Hkv * Dh).reshape(N, Hkv, Dh)
+        cnt = self.L_used * Hkv * Dh
+        self.kp = synth.qkv_block(seed, synth.STREAM_K, seq_id, cnt).reshape(-1, Hkv, Dh) if cnt else np.zeros((0, Hkv, Dh), np.float32)
+        self.vp = synth.qkv_block(seed, synth.STREAM_V, seq_id, cnt).reshape(-1, Hkv, Dh) if cnt else np.zeros((0, Hkv, Dh), np.float32)
 
     def run(self):
-        """Returns (seconds for expansion + finalise + accept, seconds for attention on self.heads)."""
+        """Seconds per stage for one step of this sequence: expansion, finalise, argmax + accept walk,
+        attention (scaled to all heads and to the full prefix)."""
         O, cfg = self.O, self.cfg
         t0 = time.perf_counter()
         tree = O.expand(self.root, self.logits_fn, self.p)
+        t1 = time.perf_counter()
         O.finalize(tree, self.L)
+        t2 = time.perf_counter()
         tt = O.target_argmax(self.target, tree.n_nodes)
         O.accept(tree, tt)
-        t1 = time.perf_counter()
+        t3 = time.perf_counter()
         g = cfg.group
         for h in self.heads:
             kv = h // g
             O.tree_attention(self.q[:, h:h + 1], self.kp[:, kv:kv + 1], self.vp[:, kv:kv + 1],
                              self.kt[:, kv:kv + 1], self.vt[:, kv:kv + 1], tree, 1.0 / math.sqrt(cfg.head_dim))
-        t2 = time.perf_counter()
-        return t1 - t0, t2 - t1
+        t4 = time.perf_counter()
+        scale = (cfg.n_q_heads / len(self.heads)) * ((self.L + cfg.budget) / (self.L_used + cfg.budget))
+        return dict(expand=t1 - t0, finalize=t2 - t1, accept=t3 - t2, attention=(t4 - t3) * scale)
 
 
-def oracle_sample_plan(cfg):
-    """Which part of a step the oracle is timed on, so that one sample stays within seconds."""
-    all_heads = cfg.n_q_heads * (cfg.prefix_max + cfg.budget) <= 32 * 4200
-    heads = list(range(cfg.n_q_heads)) if all_heads else [0, cfg.n_q_heads // 2, cfg.n_q_heads - 1]
-    return heads
-
-
-def time_oracle(cfg, seed: int, steps: int, warmup: int, budget_s: float):
-    """Times the oracle on sequence 0 of the workload.  Returns a dict with steps/s of a whole batch
-    (sequence time x batch; attention scaled from the sampled heads to all heads)."""
+def _oracle_worker(job):
+    """One host core: prepares and times the oracle on one sequence; optionally checks a tree the
+    CUDA path produced for that sequence against the oracle, layer by layer (runs in a child process)."""
+    cfg_name, seed, seq_id, steps, budget_s, gpu_tree = job
     try:
         from threadpoolctl import threadpool_limits
-        limiter = threadpool_limits(limits=1)
+        threadpool_limits(limits=1)
     except Exception:                                     # pragma: no cover
-        limiter = None
-    heads = oracle_sample_plan(cfg)
-    st = OracleStep(cfg, seed, 0, heads)
-    for _ in range(warmup):
-        st.run()
-    times = []
+        pass
+    from paper_2601_07353_b200 import synth
+    cfg = synth.CONFIGS[cfg_name]
+    st = OracleStep(cfg, seed, seq_id)
+    acc, n = dict(expand=0.0, finalize=0.0, accept=0.0, attention=0.0), 0
     t_start = time.perf_counter()
-    for i in range(steps):
-        a, b = st.run()
-        times.append(a + b * cfg.n_q_heads / len(heads))
-        if time.perf_counter() - t_start > budget_s and i + 1 >= 1:
+    for _ in range(steps):
+        r = st.run()
+        for k in acc:
+            acc[k] += r[k]
+        n += 1
+        if time.perf_counter() - t_start > budget_s:
             break
-    if limiter is not None:
-        limiter.restore_original_limits()
-    per_seq = sum(times) / len(times)
-    per_step = per_seq * cfg.batch
-    sample = (f"{len(times)} oracle steps of sequence 0 ({'all' if len(heads) == cfg.n_q_heads else len(heads)} "
-              f"of {cfg.n_q_heads} attention heads{'' if len(heads) == cfg.n_q_heads else ', scaled to all'}; "
-              f"x batch {cfg.batch})")
-    return dict(value=1.0 / per_step, unit=UNIT, cores=1, kind="oracle", sample=sample,
-                ms_per_step=per_step * 1e3, steps_timed=len(times))
+    out = {k: v / n for k, v in acc.items()}
+    out["steps"] = n
+    out["ties"] = None
+    if gpu_tree is not None:
+        # selection differences between candidates whose fp64 scores lie within 1e-5 are tolerated
+        # and counted; anything else is a mismatch
+        from tests import parity_util as PU
+        try:
+            _, tol = PU.follow_tree(cfg, st.p, st.root, st.logits_fn, gpu_tree["token"], gpu_tree["parent"],
+                                    gpu_tree["n_nodes"], gpu_tree["layer_off"], f"{cfg.name}[seq {seq_id}]")
+            out["ties"] = (tol, 0)
+        except AssertionError:
+            out["ties"] = (0, 1)
+    return out
+
+
+def time_oracle(cfg, seed: int, seq_ids, steps: int, budget_s: float, workers: int, gpu_trees=None):
+    """Times the oracle on ``seq_ids``, one sequence per host core at a time.  Returns the all-cores
+    figure (sequences run side by side), the one-core figure (mean sequence time), the per-stage
+    split and the tie count, as steps/s of a whole batch."""
+    import multiprocessing as mp
+    jobs = [(cfg.name, seed, s, steps, budget_s, None if gpu_trees is None else gpu_trees.get(s)) for s in seq_ids]
+    workers = max(1, min(workers, len(jobs)))
+    t0 = time.perf_counter()
+    if workers == 1:
+        res = [_oracle_worker(j) for j in jobs]
+    else:
+        with mp.get_context("spawn").Pool(workers) as pool:
+            res = pool.map(_oracle_worker, jobs)
+    wall = time.perf_counter() - t0
+    stages = {k: float(np.mean([r[k] for r in res])) for k in ("expand", "finalize", "accept", "attention")}
+    per_seq = sum(stages.values())                     # one core, one sequence, one step
+    one_core = 1.0 / (per_seq * cfg.batch)
+    all_cores = one_core * workers                     # `workers` sequences side by side, one core each
+    ties = [r["ties"] for r in res if r["ties"] is not None]
+    heads = oracle_heads(cfg)
+    sample = (f"{len(jobs)} sequences ({workers} at a time, one per core), {res[0]['steps']} oracle step(s) each; attention on "
+              f"{'all' if len(heads) == cfg.n_q_heads else len(heads)} of {cfg.n_q_heads} heads"
+              f"{'' if cfg.prefix_max <= ORACLE_PREFIX_SAMPLE else f' and the first {ORACLE_PREFIX_SAMPLE} prefix tokens'}"
+              f", scaled to the whole; x batch {cfg.batch}")
+    return dict(value=all_cores, unit=UNIT, cores=workers, kind="oracle", sample=sample,
+                one_core={"value": one_core, "cores": 1, "ms_per_step": per_seq * cfg.batch * 1e3},
+                stage_ms_per_sequence={k: v * 1e3 for k, v in stages.items()},
+                ties=None if not ties else {"sequences_checked": len(ties), "tolerated_within_1e-5": sum(t[0] for t in ties),
+                                            "mismatches": sum(t[1] for t in ties)},
+                setup_and_run_wall_s=wall)
 
 
 def workload_text(cfg) -> str:
@@ -220,14 +271,14 @@ def run_reference(args, cfg):
     info = dist.env_rank_info()
     if not info.is_main:
         return 0
-    r = time_oracle(cfg, args.seed, args.steps, args.warmup, budget_s=150.0)
+    cores = os.cpu_count() or 1
+    r = time_oracle(cfg, args.seed, list(range(min(cores, cfg.batch))), max(1, args.steps), 60.0, cores)
     line = {
         "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
-        "steps": r["steps_timed"], "warmup": args.warmup, "ms_per_step": r["ms_per_step"],
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / r["value"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": workload_text(cfg)},
-        "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
-                         "sample": r["sample"]},
+        "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "one_core", "stage_ms_per_sequence")},
         "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -238,7 +289,7 @@ def run_reference(args, cfg):
 # --------------------------------------------------------------------------------------------
 # the CUDA arm
 # --------------------------------------------------------------------------------------------
-def set_bytes(cfg, wl) -> int:
+def set_bytes(wl) -> int:
     """HBM bytes one step touches in one input set (upper bound: every draft row counted)."""
     t = wl.draft.numel() * 4 + wl.target.numel() * 4
     for x in (wl.q, wl.k_prefix, wl.v_prefix, wl.k_tree, wl.v_tree, wl.out):
@@ -246,24 +297,101 @@ def set_bytes(cfg, wl) -> int:
     return t
 
 
-def run_talon(args, cfg):
+def tree_statistics(cfg, sets, roofline):
+    """Algorithmic work per step and the shapes of the trees the input sets produce."""
+    B, N, V, D = cfg.batch, cfg.budget, cfg.vocab, cfg.max_depth
+    exp_b = arg_b = att_b = att_f = 0
+    n_nodes, depths, rows_per_seq = [], [], []
+    per_depth = np.zeros(D + 1)
+    for wl in sets:
+        lo = wl.tree.layer_off.cpu().numpy()
+        nn = wl.tree.n_nodes.cpu().numpy()
+        pl = wl.prefix_len.cpu().numpy()
+        dep = wl.tree.depth.cpu().numpy()
+        for b in range(B):
+            rows = roofline.expanded_rows(lo[b], N, D)
+            exp_b += roofline.expand_bytes(rows, V)
+            arg_b += roofline.argmax_bytes(int(nn[b]), V)
+            att_b += roofline.attention_bytes(int(pl[b]), int(nn[b]), cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, N)
+            att_f += roofline.attention_flops(int(pl[b]), int(nn[b]), cfg.n_q_heads, cfg.head_dim)
+            n_nodes.append(int(nn[b])); depths.append(int(dep[b, :nn[b]].max())); rows_per_seq.append(rows)
+            per_depth += np.bincount(dep[b, :nn[b]], minlength=D + 1)[:D + 1]
+    n = len(sets)
+    work = dict(expand_rows=exp_b / n, accept=arg_b / n, tree_attention=att_b / n, attention_flops=att_f / n)
+    shapes = {"n_nodes_min": min(n_nodes), "n_nodes_max": max(n_nodes), "n_nodes_mean": float(np.mean(n_nodes)),
+              "max_depth_min": min(depths), "max_depth_max": max(depths),
+              "expanded_rows_per_seq_mean": float(np.mean(rows_per_seq)),
+              "nodes_per_depth_mean": [round(float(x), 2) for x in per_depth / len(n_nodes)]}
+    return work, shapes
+
+
+def time_replays(graphs, replays: int):
+    """Milliseconds per replay: one event pair around ``replays`` back-to-back graph launches that
+    rotate over ``graphs`` (one per input set)."""
+    import torch
+    for i in range(min(3, replays)):
+        graphs[i % len(graphs)].replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(replays):
+        graphs[i % len(graphs)].replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / replays
+
+
+def kernel_pass(t, cfg, sets, stream):
+    """Times each kernel family alone.  For every input set the launches of one family are captured
+    in a CUDA graph of their own (expansion: the reset plus the D_max layer launches, since a layer
+    needs the tree the previous one left; the reset's own time is measured and subtracted); the
+    graphs are replayed back to back, rotating over the sets, between one pair of events."""
+    import torch
+    from paper_2601_07353_b200 import workload
+    D = cfg.max_depth
+    scale = 1.0 / math.sqrt(cfg.head_dim)
+    fam = {
+        "reset": lambda wl: t.reset(wl.tree, wl.root_tok, wl.prefix_len),
+        "reset+expand": lambda wl: (t.reset(wl.tree, wl.root_tok, wl.prefix_len),
+                                    [t.expand_layer(wl.tree, wl.draft) for _ in range(D)]),
+        "build_tree": lambda wl: t.build_tree(wl.tree),
+        "tree_attention": lambda wl: t.tree_attention(wl.tree, wl.q, wl.k_prefix, wl.v_prefix, wl.k_tree, wl.v_tree,
+                                                      wl.kv_start, wl.k_prefix.shape[0], cfg.n_kv_heads * cfg.head_dim,
+                                                      cfg.head_dim, wl.max_prefix_len, scale, wl.out),
+        "accept": lambda wl: t.accept(wl.tree, wl.target, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok),
+    }
+    for wl in sets:                                   # every family runs on a finished tree
+        workload.run_step(t, wl)
+    torch.cuda.synchronize()
+    out, launches = {}, {}
+    replays = max(KERNEL_REPLAYS, 2 * len(sets))
+    with torch.cuda.stream(stream):
+        for name, fn in fam.items():
+            graphs = []
+            l0 = t.launch_count()
+            for wl in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    fn(wl)
+                graphs.append(g)
+            launches[name] = (t.launch_count() - l0) / len(sets)
+            out[name] = time_replays(graphs, replays)
+            del graphs
+        for wl in sets:                               # leave every set with a complete step behind it
+            workload.run_step(t, wl)
+    torch.cuda.synchronize()
+    return out, launches, replays
+
+
+def measure(cfg, args, info, dev, dev_index, peaks, headline: bool, sampler=None):
+    """Builds the workload of ``cfg`` and measures it.  Returns the fields of a result line."""
     import torch
     from paper_2601_07353_b200 import dist, roofline, synth, talon, workload
 
-    info = dist.env_rank_info()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
-    dev_index = info.local_rank % torch.cuda.device_count()
-    torch.cuda.set_device(dev_index)
-    dev = torch.device("cuda", dev_index)
-    dist.init(info, "nccl")
-    peaks = roofline.load_peaks(ROOT)
-
     B, N, V, D = cfg.batch, cfg.budget, cfg.vocab, cfg.max_depth
     t = workload.make_talon(cfg, device=dev_index)
-    # how many input sets: bytes between two uses of a set must exceed L2 several times
     probe = workload.build_workload(cfg, t, args.seed, dist.rank_sequence_ids(info, 1, B)[0])
-    per_set = set_bytes(cfg, probe)
+    per_set = set_bytes(probe)
     n_sets = max(1, math.ceil(ROTATION_FACTOR * L2_BYTES / per_set)) if args.sets is None else args.sets
     free_b, _ = torch.cuda.mem_get_info(dev)
     n_sets = max(1, min(n_sets, int(0.6 * free_b // per_set) + 1))
@@ -271,28 +399,8 @@ def run_talon(args, cfg):
     sets = [probe] + [workload.build_workload(cfg, t, args.seed, ids[s]) for s in range(1, n_sets)]
     torch.cuda.synchronize()
     assert t.poll_status() == talon.OK
+    work, shapes = tree_statistics(cfg, sets, roofline)
 
-    # ---- per-step algorithmic work, from the trees the sets produce ----
-    exp_b = arg_b = att_b = att_f = 0
-    shapes = []
-    att_flops_set = []
-    for wl in sets:
-        f_before = att_f
-        lo = wl.tree.layer_off.cpu().numpy()
-        nn = wl.tree.n_nodes.cpu().numpy()
-        pl = wl.prefix_len.cpu().numpy()
-        for b in range(B):
-            rows = roofline.expanded_rows(lo[b], N, D)
-            exp_b += roofline.expand_bytes(rows, V)
-            arg_b += roofline.argmax_bytes(int(nn[b]), V)
-            att_b += roofline.attention_bytes(int(pl[b]), int(nn[b]), cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, N)
-            att_f += roofline.attention_flops(int(pl[b]), int(nn[b]), cfg.n_q_heads, cfg.head_dim)
-            shapes.append((int(nn[b]), int(np.max(wl.tree.depth[b].cpu().numpy())), rows))
-        att_flops_set.append(att_f - f_before)
-    per_step = {k: v / n_sets for k, v in dict(expand_rows=exp_b, target_argmax=arg_b, tree_attention=att_b).items()}
-    att_flops_step = att_f / n_sets
-
-    sampler = ClockSampler(dev_index) if info.is_main else None
     step = lambda i: workload.run_step_fused(t, sets[i % n_sets])
     # Everything below runs on a stream of its own: talon_step replays a captured graph of its
     # launches from the second call with the same arguments, which the legacy default stream cannot do.
@@ -300,51 +408,99 @@ def run_talon(args, cfg):
     main_stream = torch.cuda.Stream(dev)
     torch.cuda.set_stream(main_stream)
 
-    # ---- warm-up (every input set at least twice, so that each set's step has been captured),
-    # then an untimed pass with every kernel bracketed: which kernel dominates ----
+    # ---- warm-up: every input set at least twice, so that each set's step has been captured ----
     warm = max(args.warmup, 3, 2 * n_sets)
     for i in range(warm):
         step(i)
     torch.cuda.synchronize()
-    t.timing_enable(64 * (2 * D + 8))
-    prof_steps = args.prof_steps
-    for i in range(prof_steps):
-        step(i)
-    kt = t.timing_read()
-    kernels = {k: {"ms_per_step": ms / prof_steps, "launches_per_step": n / prof_steps} for k, (ms, n) in kt.items() if n}
-    streaming = [k for k in ("expand_rows", "tree_attention", "target_argmax") if k in kernels]
-    dominant = max(streaming, key=lambda k: kernels[k]["ms_per_step"])
-    t.timing_enable(0)
 
-    # ---- the timed region: K steps, the dominant kernel bracketed by events on the launch stream ----
+    # ---- the timed region: K steps, repeated until half a second has been measured ----
     K = args.steps
-    # the dominant kernel is bracketed on every TIMED_EVERY-th step of the timed region only, so
-    # that the event records do not slow the headline down
-    sampled = [i for i in range(K) if i % TIMED_EVERY == 0]
-    t.timing_enable(int(len(sampled) * kernels[dominant]["launches_per_step"]) + 8, [dominant])
-    launches0 = t.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    dist.barrier(info)
-    wall0 = time.time()
-    ev0.record()
-    for i in range(K):
-        t.timing_pause(i % TIMED_EVERY != 0)
-        step(i)
-    ev1.record()
-    torch.cuda.synchronize()
-    dist.barrier(info)
+    launches0 = t.launch_count()
+    reps, total, wall0 = [], 0.0, time.time()
+    max_reps = 1 if args.no_repeat else 200
+    while len(reps) < max_reps and (not reps or total < MIN_REGION_S):
+        torch.cuda.synchronize()
+        dist.barrier(info)
+        ev0.record()
+        for i in range(K):
+            step(len(reps) * K + i)
+        ev1.record()
+        torch.cuda.synchronize()
+        dist.barrier(info)
+        s = dist.max_over_ranks(ev0.elapsed_time(ev1) * 1e-3, info, dev)
+        reps.append(s)
+        total += s
     wall1 = time.time()
-    seconds = ev0.elapsed_time(ev1) * 1e-3
-    gpu_launches = t.launch_count() - launches0
-    dom_ms, dom_n = t.timing_read()[dominant]
-    t.timing_enable(0)
+    gpu_launches = (t.launch_count() - launches0) // len(reps)
     assert t.poll_status() == talon.OK
-    seconds_max = dist.max_over_ranks(seconds, info, dev)
-    value = dist.whole_job_rate(K, seconds_max, info)
+    seconds = statistics.median(reps)
+    value = dist.whole_job_rate(K, seconds, info)
+    res = {
+        "value": value, "ms_per_step": seconds / K * 1e3, "steps": K, "repeats": len(reps),
+        "spread": (max(reps) - min(reps)) / seconds if len(reps) > 1 else 0.0,
+        "warmup": warm, "warmup_requested": args.warmup, "gpu_launches": int(gpu_launches),
+        "sequence_steps_per_s": value * B, "tree_shapes": shapes,
+        "l2": f"inputs larger than L2: steps rotate over {n_sets} input sets of {per_set / 1e6:.1f} MB "
+              f"({n_sets * per_set / 1e6:.0f} MB vs 126 MB L2)",
+        "input_sets": n_sets, "timed_wall": (wall0, wall1),
+    }
+
+    # ---- each kernel family alone ----
+    ms, launches, replays = kernel_pass(t, cfg, sets, main_stream)
+    exp_ms = max(ms["reset+expand"] - ms["reset"], 1e-6)
+    gbs = lambda b, m: b / (m * 1e-3) / 1e9
+    kernels = {
+        "reset": {"ms_per_step": ms["reset"], "launches_per_step": launches["reset"]},
+        "expand_rows": {"ms_per_step": exp_ms, "launches_per_step": launches["reset+expand"] - launches["reset"],
+                        "avg_launch_us": exp_ms * 1e3 / max(1.0, launches["reset+expand"] - launches["reset"]),
+                        "algorithmic_gbs": gbs(work["expand_rows"], exp_ms)},
+        "build_tree": {"ms_per_step": ms["build_tree"], "launches_per_step": launches["build_tree"]},
+        "tree_attention": {"ms_per_step": ms["tree_attention"], "launches_per_step": launches["tree_attention"],
+                           "algorithmic_gbs": gbs(work["tree_attention"], ms["tree_attention"]),
+                           "tflops": work["attention_flops"] / (ms["tree_attention"] * 1e-3) / 1e12},
+        "accept": {"ms_per_step": ms["accept"], "launches_per_step": launches["accept"],
+                   "algorithmic_gbs": gbs(work["accept"], ms["accept"]),
+                   "note": "target argmax (the bytes) plus the accept walk (a few microseconds)"},
+    }
+    for k in ("expand_rows", "tree_attention", "accept"):
+        kernels[k]["frac_of_hbm_peak"] = kernels[k]["algorithmic_gbs"] / peaks["hbm_gbs"]
+        kernels[k]["frac_of_nominal_8tbs"] = kernels[k]["algorithmic_gbs"] / 8000.0
+    kernels["tree_attention"]["frac_of_bf16_sustained"] = kernels["tree_attention"]["tflops"] / peaks["bf16_tflops_sustained"]
+    ksum = ms["reset+expand"] + ms["build_tree"] + ms["tree_attention"] + ms["accept"]
+    res["kernels"] = kernels
+    res["kernels_sum_ms"] = ksum
+    res["kernels_sum_over_step"] = ksum / res["ms_per_step"]
+    res["kernel_timing"] = (f"each family alone: one event pair around {replays} back-to-back graph replays of its launches, "
+                            "inputs rotated over the input sets; layers that find the tree full are launched and counted")
+
+    # ---- roofline of the dominant kernel ----
+    dominant = max(("expand_rows", "tree_attention", "accept"), key=lambda k: kernels[k]["ms_per_step"])
+    kd = kernels[dominant]
+    intensity = work["attention_flops"] / max(1.0, work["tree_attention"])
+    ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    n_launch = max(1.0, kd["launches_per_step"])
+    ratio = roofline.captured_traffic_ratio(ROOT, dominant, cfg.name)
+    roof = {"kernel": dominant, "bound": "hbm", "achieved": kd["algorithmic_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": kd["frac_of_hbm_peak"], "peak_source": f"of {peaks['source']}",
+            "avg_launch_us": kd["ms_per_step"] * 1e3 / n_launch, "launches_per_step": n_launch,
+            "algorithmic_bytes_per_launch": work[dominant] / n_launch,
+            "traffic": None if ratio is None else ratio * work[dominant] / n_launch,
+            "traffic_source": None if ratio is None else "profiles/traffic_capture.json: DRAM bytes per algorithmic byte from the "
+                                                          "last ncu capture of this kernel source on this workload x this run's bytes per launch"}
+    if dominant == "tree_attention" and intensity > ridge:
+        roof.update({"bound": "tensor", "achieved": kd["tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": kd["frac_of_bf16_sustained"], "flop_per_byte": intensity, "ridge_flop_per_byte": ridge})
+    res["roofline"] = roof
+
+    if not headline:
+        t.close()
+        del sets
+        torch.cuda.empty_cache()
+        return res
 
     # ---- the same steps as one CUDA graph replay each (no library entry, no launch gaps from the host) ----
-    graph_info = None
     if not args.no_graph:
         try:
             graphs = []
@@ -355,25 +511,16 @@ def run_talon(args, cfg):
                     with torch.cuda.graph(gph, stream=side):
                         workload.run_step_fused(t, sets[s])
                     graphs.append(gph)
-            torch.cuda.synchronize()
-            for i in range(3 * n_sets):
-                graphs[i % n_sets].replay()
-            torch.cuda.synchronize()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record()
-            for i in range(K):
-                graphs[i % n_sets].replay()
-            g1.record()
-            torch.cuda.synchronize()
-            gs = dist.max_over_ranks(g0.elapsed_time(g1) * 1e-3, info, dev)
-            graph_info = {"value": dist.whole_job_rate(K, gs, info), "unit": UNIT, "ms_per_step": gs / K * 1e3}
+                torch.cuda.synchronize()
+                gms = time_replays(graphs, max(K, 3 * n_sets))
+            res["graph_replay"] = {"value": dist.whole_job_rate(1, dist.max_over_ranks(gms * 1e-3, info, dev), info),
+                                   "unit": UNIT, "ms_per_step": gms}
             del graphs
         except Exception as e:                           # graph capture is an extra, never the headline
-            graph_info = {"error": str(e).splitlines()[0][:200]}
+            res["graph_replay"] = {"error": str(e).splitlines()[0][:200]}
             torch.cuda.synchronize()
 
-    # ---- the sampling verification (the paper's temperature-1 setting) on the same trees: an extra, not the headline ----
-    sampling = None
+    # ---- the sampling verification (the paper's temperature-1 setting) on the same trees: an extra ----
     if not args.no_sampling:
         Ks = min(K, 64)
         dev_t = sets[0].target.device
@@ -399,120 +546,118 @@ def run_talon(args, cfg):
         sm_ms, sm_n = st["target_softmax_stats"]
         wk_ms, wk_n = st["accept_sample"]
         if sm_n and wk_n:
-            gbs = per_step["target_argmax"] / (sm_ms / sm_n * 1e-3) / 1e9
-            sampling = {"temperature": 1.0, "calls": Ks,
-                        "target_softmax_stats": {"ms_per_call": sm_ms / sm_n, "algorithmic_gbs": gbs,
-                                                 "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]},
-                        "accept_sample": {"ms_per_call": wk_ms / wk_n}}
+            g = work["accept"] / (sm_ms / sm_n * 1e-3) / 1e9
+            res["sampling_verify"] = {"temperature": 1.0, "calls": Ks,
+                                      "target_softmax_stats": {"ms_per_call": sm_ms / sm_n, "algorithmic_gbs": g,
+                                                               "frac_of_hbm_peak": g / peaks["hbm_gbs"],
+                                                               "note": "bracketed by events per launch"},
+                                      "accept_sample": {"ms_per_call": wk_ms / wk_n}}
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----
-    e2e = None
     if not args.no_e2e:
         pin = lambda x: x.cpu().pin_memory()
         hi32 = lambda *s: torch.zeros(*s, dtype=torch.int32).pin_memory()
-        n_host = max(1, min(n_sets, int((8 << 30) // per_set)))
+        n_host = max(1, min(n_sets, int((10 << 30) // per_set)))
         host = []
         for wl in sets[:n_host]:
             host.append((pin(wl.root_tok), pin(wl.prefix_len), pin(wl.draft), pin(wl.target), pin(wl.q),
                          pin(wl.k_prefix), pin(wl.v_prefix), pin(wl.k_tree), pin(wl.v_tree)))
         out_h = torch.zeros(B, N, cfg.n_q_heads, cfg.head_dim, dtype=torch.bfloat16).pin_memory()
-        res = (hi32(B), hi32(B, N), hi32(B, N), hi32(B, N), hi32(B, N), hi32(B), hi32(B, D + 1), hi32(B))
+        hres = (hi32(B), hi32(B, N), hi32(B, N), hi32(B, N), hi32(B, N), hi32(B), hi32(B, D + 1), hi32(B))
         h2d = sum(x.numel() * x.element_size() for x in host[0]) + 8 * B
-        d2h = out_h.numel() * 2 + sum(x.numel() * 4 for x in res)
-        Ke = max(3, min(K, int(20.0 / max(1e-4, h2d / 20e9))))       # keep this leg within ~20 s
+        d2h = out_h.numel() * 2 + sum(x.numel() * 4 for x in hres)
+        Ke = max(3, min(K, int(8.0 / max(1e-4, h2d / 20e9))))       # keep this leg within ~10 s
         scale = 1.0 / math.sqrt(cfg.head_dim)
-        for i in range(3):
-            assert t.step_host(*host[i % n_host], scale, out_h, *res) == talon.OK
+        for i in range(2):
+            assert t.step_host(*host[i % n_host], scale, out_h, *hres) == talon.OK
         torch.cuda.synchronize()
         dist.barrier(info)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         w0 = time.perf_counter()
         e0.record()
         for i in range(Ke):
-            t.step_host(*host[i % n_host], scale, out_h, *res)
+            t.step_host(*host[i % n_host], scale, out_h, *hres)
         e1.record()
         torch.cuda.synchronize()
         w1 = time.perf_counter()
         dist.barrier(info)
         es = dist.max_over_ranks(max(e0.elapsed_time(e1) * 1e-3, 0.0), info, dev)
-        e2e = {"value": dist.whole_job_rate(Ke, es, info), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": Ke, "ms_per_step": es / Ke * 1e3,
-               "host_wall_ms_per_step": (w1 - w0) / Ke * 1e3,
-               "api": "talon_step_host (pinned host buffers in, host results out)"}
+        res["e2e"] = {"value": dist.whole_job_rate(Ke, es, info), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "steps": Ke, "ms_per_step": es / Ke * 1e3,
+                      "host_wall_ms_per_step": (w1 - w0) / Ke * 1e3,
+                      "api": "talon_step_host (pinned host buffers in, host results out)"}
         del host
 
+    # ---- the oracle beside it, on the machine's host cores, and the tie count against the CUDA trees ----
+    if info.is_main and info.world == 1 and not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        gpu_trees, seqs = {}, []
+        for wl in sets:
+            tok, par = wl.tree.token.cpu().numpy(), wl.tree.parent.cpu().numpy()
+            nn, lo = wl.tree.n_nodes.cpu().numpy(), wl.tree.layer_off.cpu().numpy()
+            for bi, sid in enumerate(wl.seq_ids):
+                if len(seqs) < cores:
+                    seqs.append(sid)
+                    gpu_trees[sid] = dict(token=tok[bi], parent=par[bi], n_nodes=int(nn[bi]), layer_off=lo[bi])
+        r = time_oracle(cfg, args.seed, seqs, 1, 20.0, cores, gpu_trees)
+        res["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "one_core",
+                                                 "stage_ms_per_sequence", "setup_and_run_wall_s")}
+        res["selection_ties"] = r["ties"]
+    t.close()
+    del sets
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_talon(args):
+    import torch
+    from paper_2601_07353_b200 import dist, roofline, synth
+
+    info = dist.env_rank_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    dev_index = info.local_rank % torch.cuda.device_count()
+    torch.cuda.set_device(dev_index)
+    dev = torch.device("cuda", dev_index)
+    dist.init(info, "nccl")
+    peaks = roofline.load_peaks(ROOT)
+    head_name = args.config or HEADLINE
+    subs = [] if (args.config or args.no_sub_configs or info.world > 1) else SUB_CONFIGS
+
+    sampler = ClockSampler(dev_index) if info.is_main else None
+    head = measure(synth.CONFIGS[head_name], args, info, dev, dev_index, peaks, True)
+    wall0, wall1 = head.pop("timed_wall")
+    clocks = sampler.summary(wall0, wall1) if sampler is not None else None
+    others = {}
+    for name in subs:
+        torch.cuda.set_stream(torch.cuda.default_stream(dev))
+        r = measure(synth.CONFIGS[name], args, info, dev, dev_index, peaks, False)
+        r.pop("timed_wall")
+        others[name] = {"workload": workload_text(synth.CONFIGS[name]),
+                        **{k: r[k] for k in ("value", "ms_per_step", "steps", "repeats", "spread", "roofline", "kernels",
+                                             "kernels_sum_over_step", "tree_shapes", "input_sets", "gpu_launches")}}
     if sampler is not None:
         sampler.stop()
-    clocks = sampler.summary(wall0, wall1) if sampler is not None else None
-
-    # ---- roofline of the dominant kernel over the timed region ----
-    per_set_bytes = []
-    for wl in sets:
-        lo = wl.tree.layer_off.cpu().numpy(); nn = wl.tree.n_nodes.cpu().numpy(); pl = wl.prefix_len.cpu().numpy()
-        tot = 0
-        for b in range(B):
-            if dominant == "expand_rows":
-                tot += roofline.expand_bytes(roofline.expanded_rows(lo[b], N, D), V)
-            elif dominant == "target_argmax":
-                tot += roofline.argmax_bytes(int(nn[b]), V)
-            else:
-                tot += roofline.attention_bytes(int(pl[b]), int(nn[b]), cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, N)
-        per_set_bytes.append(tot)
-    dom_bytes_total = float(sum(per_set_bytes[i % n_sets] for i in sampled))      # the bracketed steps' bytes
-    dom_flops_total = float(sum(att_flops_set[i % n_sets] for i in sampled))
-    roof = None
-    if dom_n > 0 and dom_ms > 0:
-        timed_frac = dom_n / max(1.0, len(sampled) * kernels[dominant]["launches_per_step"])
-        achieved = dom_bytes_total * timed_frac / (dom_ms * 1e-3) / 1e9
-        intensity = att_flops_step / max(1.0, per_step["tree_attention"])
-        ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-        bound = "hbm"
-        ratio = roofline.captured_traffic_ratio(dominant)
-        roof = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                "traffic": None if ratio is None else ratio * dom_bytes_total * timed_frac / dom_n,
-                "traffic_source": None if ratio is None else "ncu capture of an earlier run, same kernel source: DRAM bytes per algorithmic byte x this run's bytes per launch",
-                "launches_timed": int(dom_n), "timed_steps": f"1 step in {TIMED_EVERY} of the timed region", "avg_launch_us": dom_ms / dom_n * 1e3,
-                "algorithmic_bytes_per_launch": dom_bytes_total * timed_frac / dom_n}
-        if dominant == "tree_attention" and intensity > ridge:
-            tf = dom_flops_total * timed_frac / (dom_ms * 1e-3) / 1e12
-            roof.update({"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": tf / peaks["bf16_tflops_sustained"]})
-    # secondary figures from the bracketed pass (event pairs around every kernel; launch gaps included)
-    for k in ("expand_rows", "target_argmax", "tree_attention"):
-        if k in kernels and kernels[k]["ms_per_step"] > 0:
-            kernels[k]["algorithmic_gbs"] = per_step[k] / (kernels[k]["ms_per_step"] * 1e-3) / 1e9
-            kernels[k]["frac_of_hbm_peak"] = kernels[k]["algorithmic_gbs"] / peaks["hbm_gbs"]
-            kernels[k]["frac_of_nominal_8tbs"] = kernels[k]["algorithmic_gbs"] / 8000.0
-    if "tree_attention" in kernels:
-        kernels["tree_attention"]["tflops"] = att_flops_step / (kernels["tree_attention"]["ms_per_step"] * 1e-3) / 1e12
-
-    cpu = None
-    if info.is_main and info.world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(cfg, args.seed, 10, 0, budget_s=15.0)
-        cpu = {"value": r["value"], "unit": UNIT, "cores": r["cores"], "kind": "oracle", "sample": r["sample"]}
 
     if info.is_main:
-        nn = [s[0] for s in shapes]; dp = [s[1] for s in shapes]
+        cfg = synth.CONFIGS[head_name]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": info.world, "steps": K, "warmup": warm,
-            "ms_per_step": seconds_max / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32 logits, f64 path scores, bf16 attention (f32 accumulate)", "data": "synthetic",
-            "config": {"workload": workload_text(cfg),
-                       "l2": f"inputs larger than L2: steps rotate over {n_sets} input sets of {per_set / 1e6:.1f} MB "
-                             f"({n_sets * per_set / 1e6:.0f} MB vs 126 MB L2)",
-                       "step": f"talon_step: reset + {D} expand-layer calls + build + tree attention + accept "
-                               "(the library replays its own captured graph of these launches; steps whose "
-                               "dominant kernel is bracketed by events are launched one by one)",
-                       "sequences_per_rank": B, "input_sets": n_sets},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(gpu_launches), "roofline": roof, "cpu_baseline": cpu,
-            "graph_replay": graph_info, "kernels": kernels, "sampling_verify": sampling,
-            "tree_shapes": {"n_nodes_min": min(nn), "n_nodes_max": max(nn), "max_depth_min": min(dp), "max_depth_max": max(dp),
-                            "expanded_rows_per_seq_mean": float(np.mean([s[2] for s in shapes]))},
-            "sequence_steps_per_s": value * B,
+            "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": info.world, "steps": head["steps"],
+            "warmup": head["warmup"], "warmup_requested": head["warmup_requested"], "ms_per_step": head["ms_per_step"],
+            "repeats": head["repeats"], "spread": head["spread"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+            "config": {"workload": workload_text(cfg), "l2": head["l2"],
+                       "step": f"talon_step: reset + {cfg.max_depth} expand-layer calls + build + tree attention + accept "
+                               "(the library replays its own captured graph of these launches)",
+                       "sequences_per_rank": cfg.batch, "input_sets": head["input_sets"]},
+            "clocks": clocks, "e2e": head.get("e2e"), "gpu_launches": head["gpu_launches"], "roofline": head["roofline"],
+            "cpu_baseline": head.get("cpu_baseline"), "selection_ties": head.get("selection_ties"),
+            "graph_replay": head.get("graph_replay"), "kernels": head["kernels"], "kernel_timing": head["kernel_timing"],
+            "kernels_sum_over_step": head["kernels_sum_over_step"], "sampling_verify": head.get("sampling_verify"),
+            "tree_shapes": head["tree_shapes"], "sequence_steps_per_s": head["sequence_steps_per_s"],
+            "configs": others,
         }
         print(json.dumps(line))
-    t.close()
     dist.shutdown()
     return 0
 
@@ -576,14 +721,16 @@ def main(argv=None):
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["talon", "reference"], default="talon")
-    ap.add_argument("--config", default="llama8b")
+    ap.add_argument("--config", default=None,
+                    help=f"measure this workload only (default: {HEADLINE} as the headline, the others under 'configs')")
     ap.add_argument("--seed", type=int, default=None)
     ap.add_argument("--sets", type=int, default=None, help="input sets to rotate over (default: enough to defeat L2)")
-    ap.add_argument("--prof-steps", type=int, default=32, help="steps of the untimed per-kernel pass")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sampling", action="store_true", help="skip the sampling-verification extra")
+    ap.add_argument("--no-sub-configs", action="store_true", help="skip the other workloads")
+    ap.add_argument("--no-repeat", action="store_true", help="time the K steps once, however short")
     ap.add_argument("--zipf-micro", action="store_true",
                     help="instead of the step benchmark: single-layer expansion latency on Zipf rows")
     args = ap.parse_args(argv)
@@ -592,14 +739,13 @@ def main(argv=None):
         args.seed = synth.DEFAULT_SEED
     if args.zipf_micro:
         return run_zipf_micro(args)
-    cfg = synth.CONFIGS[args.config]
     if args.impl == "reference":
-        args.steps = 10 if args.steps is None else args.steps
-        args.warmup = 1 if args.warmup is None else args.warmup
-        return run_reference(args, cfg)
-    args.steps = 2000 if args.steps is None else args.steps
-    args.warmup = 20 if args.warmup is None else args.warmup
-    return run_talon(args, cfg)
+        args.steps = 1 if args.steps is None else args.steps
+        args.warmup = 0 if args.warmup is None else args.warmup
+        return run_reference(args, synth.CONFIGS[args.config or HEADLINE])
+    args.steps = 100 if args.steps is None else args.steps
+    args.warmup = 5 if args.warmup is None else args.warmup
+    return run_talon(args)
 
 
 if __name__ == "__main__":

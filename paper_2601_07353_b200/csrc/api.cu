@@ -115,6 +115,10 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     const char *mt = std::getenv("TALON_ATTN_MIN_TILES");
     c->attn_min_tiles = mt ? std::atoi(mt) : 2;
     if (c->attn_min_tiles < 1) c->attn_min_tiles = 1;
+    const char *ms = std::getenv("TALON_EXPAND_MAX_SPLIT");
+    c->expand_max_split = ms ? std::atoi(ms) : talon::FX_MAX_SPLITS - 1;
+    if (c->expand_max_split < 1) c->expand_max_split = 1;
+    if (c->expand_max_split > talon::FX_MAX_SPLITS - 1) c->expand_max_split = talon::FX_MAX_SPLITS - 1;
     const char *e = std::getenv("TALON_PDL");
     c->pdl = !e ? -1 : (e[0] == '1' ? 1 : 0);
     const char *g = std::getenv("TALON_STEP_GRAPH");
@@ -136,6 +140,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
   alloc((void **)&c->d_part_ms, sizeof(float2) * (size_t)c->items_cap);
   alloc((void **)&c->d_row_keys, sizeof(unsigned long long) * (size_t)c->rows_cap * c->key_stride);
   alloc((void **)&c->d_row_lse, sizeof(double) * (size_t)c->rows_cap);
+  alloc((void **)&c->d_row_score, sizeof(double) * (size_t)c->rows_cap * c->key_stride);
   alloc((void **)&c->d_row_count, sizeof(unsigned int) * (size_t)c->rows_cap);
   alloc((void **)&c->d_seq_count, sizeof(unsigned int) * (size_t)p->batch_max);
   alloc((void **)&c->d_argmax, sizeof(unsigned long long) * nrow);
@@ -167,7 +172,7 @@ talon_status talon_destroy(talon_ctx *c) {
   if (!c) return TALON_OK;
   cudaSetDevice(c->device);
   cudaFree(c->d_status); cudaFree(c->d_prefix_len); cudaFree(c->d_part_keys); cudaFree(c->d_part_ms);
-  cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_count); cudaFree(c->d_seq_count); cudaFree(c->d_argmax);
+  cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_score); cudaFree(c->d_row_count); cudaFree(c->d_seq_count); cudaFree(c->d_argmax);
   cudaFree(c->d_target_tok); cudaFree(c->d_samp_ms); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
   talon_timing_enable(c, 0, 0u);

@@ -2,22 +2,32 @@
 // for per-parent candidate caps k <= 32 (the usual case: the paper's K is 10).
 //
 // Streaming phase.  The frontier's fp32 logit rows are cut into equal chunks, one CTA per chunk
-// at a time.  In a single read of its chunk a CTA produces the chunk's share of the softmax
-// normaliser of Eq. 3 (maximum and sum of exponentials) and the chunk's k largest logits with
-// their token ids.
-//   * A chunk of at most 4096 elements sits in registers (16 per thread).  The smallest of the
-//     256/G maxima of G-lane groups bounds the chunk's k-th largest element from below (the
-//     groups hold 256/G >= k different elements that large), so only elements at or above it
-//     go to a shared pool, which is then ranked by counting.
-//   * A longer chunk is streamed tile by tile; each warp keeps a sorted list of its best k
-//     keys across its lanes plus a queue of elements that passed the current threshold, and a
-//     full queue is folded into the list with a bitonic sort and merge.
+// at a time, and a chunk into eight slices, one per warp.  A warp streams its slice on its own:
+// 2 KB bulk copies (TMA, no multicast) into a private ring of shared-memory slots with private
+// mbarriers, so no CTA-wide barrier sits on the streaming path.  In the single read of its slice
+// a warp produces
+//   * its share of the softmax normaliser of Eq. 3 (per-lane running maximum and sum of
+//     exponentials), and
+//   * an unsorted buffer of every element that reached the warp's threshold.  The threshold is a
+//     lower bound of the row's k-th largest logit that only grows: the k-th largest of the 32
+//     per-lane running maxima (k different elements that large have been seen), refreshed after
+//     tiles 1, 2, 4, 8, ...; the smallest of the eight warps' ceil(k/8)-th largest lane maxima
+//     (again k different elements); and, on gated layers, the running maximum plus ln(mu): by
+//     Eq. 4 a candidate can only survive if its path score is within ln(mu) of the layer's best,
+//     which is at least the best of its own row, so a logit more than |ln(mu)| below the row
+//     maximum never matters.  Nothing is sorted while streaming; a buffer that fills up is cut
+//     back to its k largest keys.
+// At the end of a chunk the eight buffers meet in a CTA pool that is ranked by counting, and the
+// chunk's k best keys and normaliser go to global memory.
 //
-// Selection phase.  The CTA that finishes the last chunk of a sequence merges that sequence's
-// chunk results into per-row top-k lists and log-sum-exps, scores the pooled candidates with
-// log p(u) = log p(v) + log P(w | v) (Eq. 2-3), applies Top-K (Eq. 5) or the confidence gate
-// p(u) >= mu * max p (Eq. 4), truncates to the remaining budget, and appends the survivors with
-// parent links, depths, scores and ancestor-mask rows.  Nothing returns to the host in between.
+// Selection phase.  Frontiers of at most eight rows: the CTA that finishes a sequence's last chunk
+// merges that sequence's rows, one warp per row.  Wider frontiers: the CTA that finishes a row's
+// last chunk merges that row (rows of one sequence finish all over the grid, so the merges run in
+// parallel), and the CTA that finishes the sequence's last row collects the row results.  Either
+// way that CTA then scores the pooled candidates with log p(u) = log p(v) + log P(w | v)
+// (Eq. 2-3), applies Top-K (Eq. 5) or the confidence gate p(u) >= mu * max p (Eq. 4), truncates
+// to the remaining budget, and appends the survivors with parent links, depths, scores and
+// ancestor-mask rows.  Nothing returns to the host in between.
 #include <cuda/atomic>
 #include <math_constants.h>
 
@@ -31,18 +41,29 @@ constexpr unsigned FULL = 0xFFFFFFFFu;
 constexpr float LOG2E_F = 1.4426950408889634f;
 typedef unsigned long long u64;
 
+constexpr int XS_WTILE = 512;                 // floats a warp takes per step: 16 per lane, one 2 KB copy
+constexpr int XS_RING = 3;                    // copies in flight per warp
+constexpr int XS_BUF = FX_QCAP;               // keys a warp's candidate buffer holds
+constexpr int XS_POOL = 512;                  // keys the CTA pool holds
+constexpr int XS_TWO_LEVEL = EXP_WARPS;       // frontiers wider than this merge their rows all over the grid
+static_assert(XS_WTILE * EXP_WARPS == EXP_TILE, "a CTA step is eight warp tiles");
+static_assert(XS_BUF >= 64 && XS_POOL >= EXP_WARPS * 32, "buffers must hold a cut-back list plus one ballot");
+
 struct FusedArgs {
   const float *logits;
   int64_t row_stride;
   int rows_per_seq, layout;
   talon_tree t;
   int lo_stride;
-  int B, N, W, V, d, k, key_stride, target_items, max_splits, items_cap;
+  int B, N, W, V, d, k, key_stride, max_split;
   int root_topk, init_layers;
   double log_mu;
   u64 *part_keys;          // [items, key_stride]  per-chunk top-k, descending
   float2 *part_ms;         // [items]              per-chunk (max, sum of exp)
-  unsigned int *seq_count; // [B]                  chunks finished per sequence (zero between layers)
+  u64 *row_keys;           // [rows, key_stride]   per-row top-k (wide frontiers)
+  double *row_score;       // [rows, key_stride]   log p(u) of those candidates; slot 0 NaN: row not finite
+  unsigned int *row_count; // [rows]               chunks finished per row (zero between layers)
+  unsigned int *seq_count; // [B]                  chunks or rows finished per sequence (zero between layers)
   int *status;
 };
 
@@ -53,7 +74,31 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// ---- bulk-copy ring: a longer chunk is brought in by the TMA engine, FX_RING tiles ahead ----
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ u64 pack_f32x2(float lo, float hi) {
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack_f32x2(u64 v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma_f32x2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// ---- bulk-copy ring ----
 __device__ inline uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ inline void ring_bar_init(uint32_t bar) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
@@ -107,6 +152,20 @@ __device__ inline u64 warp_sort_desc(u64 x, int lane) {
   return x;
 }
 
+// the same for one float per lane (NaN never appears: the inputs are maxima taken with fmaxf)
+__device__ inline float warp_sort_desc_f32(float x, int lane) {
+#pragma unroll
+  for (int sz = 2; sz <= 32; sz <<= 1) {
+#pragma unroll
+    for (int j = sz >> 1; j > 0; j >>= 1) {
+      const float o = __shfl_xor_sync(FULL, x, j);
+      const bool keep_max = (((lane & j) == 0) == ((lane & sz) == 0));
+      x = keep_max ? fmaxf(x, o) : fminf(x, o);
+    }
+  }
+  return x;
+}
+
 // list (descending across lanes) <- the 32 largest of list U q, q unsorted
 __device__ inline u64 warp_merge_desc(u64 list, u64 q, int lane) {
   q = warp_sort_desc(q, lane);
@@ -119,60 +178,11 @@ __device__ inline u64 warp_merge_desc(u64 list, u64 q, int lane) {
   return x;
 }
 
-// Folds the first 32 queued keys into the warp's list, moves the rest of the queue (up to
-// FX_QCAP - 32 keys) to its front and raises the threshold to the list's k-th key.
-__device__ __forceinline__ void fold_queue(u64 &list, int &qn, float &thr_f, u64 *queue, float thr0, int k,
-                                           int lane) {
-  list = warp_merge_desc(list, queue[lane], lane);
-  const int rem = qn - 32;
-  const u64 r0 = queue[32 + lane], r1 = queue[64 + lane], r2 = queue[96 + lane];
-  __syncwarp();
-  if (lane < rem) queue[lane] = r0;
-  if (32 + lane < rem) queue[32 + lane] = r1;
-  if (64 + lane < rem) queue[64 + lane] = r2;
-  __syncwarp();
-  qn = rem;
-  const u64 kth = shfl_u64(list, k - 1);
-  if (kth) thr_f = fmaxf(thr0, key_logit(kth));
-}
-
-// Makes a warp's threshold known to the other warps of the CTA (monotone: a maximum).
-__device__ __forceinline__ void publish_thr(unsigned *thr_cta, float thr_f, int lane) {
-  if (lane == 0 && thr_f > -CUDART_INF_F) atomicMax(thr_cta, f32_ord(thr_f));
-}
-
-// Folds a queue of fewer than 32 keys into the list (queue left empty).
-__device__ __forceinline__ void flush_queue(u64 &list, int &qn, float &thr_f, const u64 *queue, float thr0, int k,
-                                            int lane) {
-  list = warp_merge_desc(list, lane < qn ? queue[lane] : 0ull, lane);
-  qn = 0;
-  const u64 kth = shfl_u64(list, k - 1);
-  if (kth) thr_f = fmaxf(thr0, key_logit(kth));
-}
-
 // Exclusive scan of the per-sequence frontier sizes: s_base[b] = first packed row of sequence
-// b, s_base[B] = total rows.  A sequence whose tree is full has no rows.
+// b, s_base[B] = total rows.  A sequence whose tree is full has no rows.  The tree's size before
+// this layer is layer_off[d + 1], which this launch never writes (n_nodes changes under it).
 __device__ void frontier_bases(const FusedArgs &a, int *s_base, int *s_warp) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (a.B <= 32) {
-    if (warp == 0) {
-      int f = 0;
-      if (lane < a.B && a.t.n_nodes[lane] < a.N) {
-        f = a.t.layer_off[lane * a.lo_stride + a.d + 1] - a.t.layer_off[lane * a.lo_stride + a.d];
-        f = max(f, 0);
-      }
-      int inc = f;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(FULL, inc, o);
-        if (lane >= o) inc += t;
-      }
-      if (lane < a.B) s_base[lane] = inc - f;
-      if (lane == a.B - 1) s_base[a.B] = inc;
-    }
-    __syncthreads();
-    return;
-  }
   constexpr int PER = (MAX_BATCH + EXP_THREADS - 1) / EXP_THREADS;
   int f[PER];
   int sum = 0;
@@ -180,9 +190,9 @@ __device__ void frontier_bases(const FusedArgs &a, int *s_base, int *s_warp) {
   for (int i = 0; i < PER; ++i) {
     const int b = tid * PER + i;
     int v = 0;
-    if (b < a.B && a.t.n_nodes[b] < a.N) {
-      v = a.t.layer_off[b * a.lo_stride + a.d + 1] - a.t.layer_off[b * a.lo_stride + a.d];
-      v = max(v, 0);
+    if (b < a.B) {
+      const int lo = a.t.layer_off[b * a.lo_stride + a.d], hi = a.t.layer_off[b * a.lo_stride + a.d + 1];
+      v = hi < a.N ? max(hi - lo, 0) : 0;
     }
     f[i] = v;
     sum += v;
@@ -235,34 +245,51 @@ __device__ inline double f64_unord(u64 o) {
   return __longlong_as_double((long long)b);
 }
 
-// Chunks per row for this layer.  Every CTA of the grid is resident, so a layer takes
-// ceil(items / grid) rounds of one chunk each: the cost of a candidate split count is
-// rounds x (tiles per chunk + a fixed per-chunk overhead of about two tiles).  Chunks of one
-// row are equal up to rounding to 4 elements (rows are 16-byte aligned), and a split row keeps
-// at least 1024 elements per chunk so that every warp of a CTA holds some.  Lane l scores the
-// split count l + 1; the warp keeps the cheapest (the smaller count on ties).
-__device__ inline LayerGeom balanced_geom(int total_rows, int vocab, int grid, int max_splits, int items_cap) {
-  const int lane = threadIdx.x & 31;
-  unsigned best = 0xFFFFFFFFu;               // cost << 8 | splits
-  if (total_rows > 0) {
-    const int sp = lane + 1;
-    int len = (((vocab + sp - 1) / sp) + 3) & ~3;
-    const int eff = (vocab + len - 1) / len;
-    const bool fits = sp == 1 || (sp <= max_splits && len >= 1024 && (long long)total_rows * eff <= items_cap);
-    if (fits) {
-      const int rounds = (total_rows * eff + grid - 1) / grid;
-      const unsigned cost = (unsigned)rounds * (unsigned)(2 * ((len + EXP_TILE - 1) / EXP_TILE) + 4);
-      best = (min(cost, 0xFFFFFFu) << 8) | (unsigned)eff;
-    }
+// How a layer is cut.  The frontier's rows are laid end to end on a line, `pitch` elements apart,
+// and the CTAs of the grid take consecutive spans of `span` elements of that line (both multiples
+// of four: rows are 16-byte aligned).
+//   * Few rows (the grid holds at least two CTAs per row): a row is cut into S equal chunks, one
+//     CTA each, S as large as the grid allows (at most FX_MAX_SPLITS - 1, at least 4096 elements
+//     per chunk); pitch = S * span, so no span crosses a row.
+//   * Many rows: pitch is the row length and every CTA takes the same share of the whole line, so
+//     every CTA (and every SM) streams the same number of bytes whatever the number of rows; a span
+//     that crosses a row boundary is worked off as one chunk per row it touches.
+// Either way a row has at most FX_MAX_SPLITS chunks (one lane per chunk in the merge).  Chunk
+// results live at index (CTA + packed row), which grows along the line; a row's chunks are
+// consecutive there.
+struct SpanGeom {
+  unsigned span;       // elements of the line per CTA
+  unsigned pitch;      // elements of the line per row (>= the row length)
+};
+
+__device__ inline unsigned div_u64(unsigned long long a, unsigned b) {
+  return a <= 0xFFFFFFFFull ? (unsigned)a / b : (unsigned)(a / b);
+}
+
+__device__ inline SpanGeom span_geom(int total_rows, int vocab, int grid, int max_split) {
+  SpanGeom g;
+  const unsigned vp = ((unsigned)vocab + 3u) & ~3u;
+  const unsigned per_row = total_rows > 0 ? (unsigned)grid / (unsigned)total_rows : 1u;
+  if (per_row >= 2u) {
+    const unsigned S = max(1u, min(min(per_row, (unsigned)max_split), vp / 4096u));
+    g.span = ((vp + S - 1u) / S + 3u) & ~3u;
+    g.pitch = S * g.span;
+  } else {
+    const unsigned long long line = (unsigned long long)total_rows * vp;
+    const unsigned span = (div_u64(line + grid - 1, (unsigned)grid) + 3u) & ~3u;
+    const unsigned span_min = max(4096u, ((vp + FX_MAX_SPLITS - 2) / (FX_MAX_SPLITS - 1) + 3u) & ~3u);
+    g.span = max(span, span_min);
+    g.pitch = vp;
   }
-#pragma unroll
-  for (int o = 16; o; o >>= 1) best = min(best, __shfl_xor_sync(FULL, best, o));
-  LayerGeom g;
-  g.total_rows = total_rows;
-  g.splits = total_rows > 0 ? (int)(best & 0xFFu) : 1;
-  g.chunk_len = (((vocab + g.splits - 1) / g.splits) + 3) & ~3;
-  g.splits = (vocab + g.chunk_len - 1) / g.chunk_len;
   return g;
+}
+
+// First chunk-result index and number of chunks of packed row `row`.
+__device__ inline void row_chunks(const SpanGeom &g, int row, int &item0, int &S) {
+  const unsigned long long lo = (unsigned long long)row * g.pitch;
+  const unsigned first = div_u64(lo, g.span), last = div_u64(lo + g.pitch - 1, g.span);
+  item0 = (int)first + row;
+  S = (int)(last - first) + 1;
 }
 
 // Where a packed frontier row lives: sequence, index inside that sequence's frontier, tree
@@ -300,179 +327,221 @@ __device__ inline RowLoc locate_row(const FusedArgs &a, const Frontier &fr, int 
   return r;
 }
 
-// Shared-memory carve-up of the selection phase.
+// ---------------------------------------------------------------------------------------
+// Streaming state of one warp
+// ---------------------------------------------------------------------------------------
+struct WarpStream {
+  float m_t, s_t;        // this lane's running maximum and sum of exponentials relative to it
+  float thr_f;           // an element below it cannot be among the row's k best (warp-uniform)
+  u64 thr_key;           // after a cut-back: the buffer's k-th key; only larger keys enter (warp-uniform)
+  int cnt;               // keys in the warp's buffer (warp-uniform)
+};
+
+// Cuts the warp's buffer back to its (at most) ke largest keys, sorted descending at the front,
+// and raises the thresholds to the ke-th of them when there are that many.
+struct CutBack { u64 thr_key; float thr_f; int cnt; };
+__device__ __noinline__ CutBack cut_back_impl(u64 *buf, int ke, int n, float thr_f, u64 thr_key) {
+  const int lane = threadIdx.x & 31;
+  u64 list = 0ull;
+  for (int off = 0; off < n; off += 32) list = warp_merge_desc(list, off + lane < n ? buf[off + lane] : 0ull, lane);
+  __syncwarp();
+  const bool keep = lane < ke && list != 0ull;
+  if (keep) buf[lane] = list;
+  CutBack r;
+  r.cnt = __popc(__ballot_sync(FULL, keep));
+  r.thr_key = thr_key;
+  r.thr_f = thr_f;
+  const u64 kth = shfl_u64(list, ke - 1);
+  if (kth != 0ull) {
+    r.thr_key = kth;
+    r.thr_f = fmaxf(thr_f, key_logit(kth));
+  }
+  __syncwarp();
+  return r;
+}
+__device__ __forceinline__ void cut_back(u64 *buf, int ke, WarpStream &w, int lane) {
+  (void)lane;
+  const CutBack r = cut_back_impl(buf, ke, w.cnt, w.thr_f, w.thr_key);
+  w.cnt = r.cnt; w.thr_key = r.thr_key; w.thr_f = r.thr_f;
+}
+
+// Raises the warp's threshold from what it has seen so far (see the header of this file).
+// s_wtop[w] holds warp w's (share_pos + 1)-th largest lane maximum, s_wmax[w] its largest.
+__device__ __forceinline__ void refresh_threshold(WarpStream &w, int ke, int share_pos, bool gated, float ln_mu,
+                                                  float *s_wtop, float *s_wmax, int lane, int warp) {
+  float cand, wmax, mine;
+  if (share_pos == 0) {
+    // ke <= 8: the eight 4-lane groups hold eight different elements at least as large as the
+    // smallest group maximum; the warp maximum is what the other warps get to see
+    float g = fmaxf(w.m_t, __shfl_xor_sync(FULL, w.m_t, 1));
+    g = fmaxf(g, __shfl_xor_sync(FULL, g, 2));
+    float hi = g, lo = g;
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      hi = fmaxf(hi, __shfl_xor_sync(FULL, hi, o));
+      lo = fminf(lo, __shfl_xor_sync(FULL, lo, o));
+    }
+    cand = lo; wmax = hi; mine = hi;
+  } else {
+    const float sorted = warp_sort_desc_f32(w.m_t, lane);
+    cand = __shfl_sync(FULL, sorted, ke - 1);
+    wmax = __shfl_sync(FULL, sorted, 0);
+    mine = __shfl_sync(FULL, sorted, share_pos);
+  }
+  if (lane == 0) { s_wtop[warp] = mine; s_wmax[warp] = wmax; }
+  __syncwarp();
+  // eight warps x (share_pos + 1) lane maxima >= the smallest published value: at least ke elements
+  float omin = lane < EXP_WARPS ? s_wtop[lane] : CUDART_INF_F;
+  float omax = lane < EXP_WARPS ? s_wmax[lane] : -CUDART_INF_F;
+#pragma unroll
+  for (int o = 4; o; o >>= 1) {
+    omin = fminf(omin, __shfl_xor_sync(FULL, omin, o));
+    omax = fmaxf(omax, __shfl_xor_sync(FULL, omax, o));
+  }
+  omin = __shfl_sync(FULL, omin, 0);
+  omax = fmaxf(wmax, __shfl_sync(FULL, omax, 0));
+  cand = fmaxf(cand, omin);
+  if (gated && omax > -CUDART_INF_F) {
+    // fp32 rounding of the sum and of ln(mu), and the 1e-5 band around the gate, stay inside the slack
+    cand = fmaxf(cand, omax + ln_mu - (1e-4f + 1e-6f * fabsf(omax)));
+  }
+  w.thr_f = fmaxf(w.thr_f, cand);
+}
+
+// Appends the elements of one tile that reach the threshold to the warp's buffer.  `slot` is the
+// warp's copy of the tile in shared memory (still intact: it is refilled after this call), tok_tile
+// the token id of its first element; lane l holds elements (i / 4) * 128 + l * 4 + i % 4 of it in v.
+__device__ __forceinline__ void collect_tile(const float *slot, const float (&v)[16], int tok_tile, int ke, u64 *buf,
+                                             WarpStream &w, int lane) {
+  unsigned mm = 0u;
+#pragma unroll
+  for (int i = 0; i < 16; ++i)
+    if (v[i] >= w.thr_f) mm |= 1u << i;
+  const int c = __popc(mm);
+  int inc = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(FULL, inc, o);
+    if (lane >= o) inc += t;
+  }
+  const int total = __shfl_sync(FULL, inc, 31);
+  if (w.thr_key == 0ull && w.cnt + total <= XS_BUF) {
+    // the usual case: a handful of elements in a few lanes; each lane fetches its own from the slot
+    int pos = w.cnt + inc - c;
+    while (mm) {
+      const int i = __ffs(mm) - 1;
+      mm &= mm - 1u;
+      const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
+      buf[pos++] = cand_key(slot[e], (uint32_t)(tok_tile + e));
+    }
+    w.cnt += total;
+    __syncwarp();
+    if (w.cnt > XS_BUF - 32) cut_back(buf, ke, w, lane);
+    return;
+  }
+  // After a cut-back only keys above the buffer's k-th enter, and more may arrive than the buffer
+  // holds (equal logits, a sorted row, a cold threshold): take the tile one register slot at a
+  // time, cutting back whenever a ballot's worth might not fit.
+  if (w.cnt + total > XS_BUF) cut_back(buf, ke, w, lane);
+#pragma unroll 1
+  for (int i = 0; i < 16; ++i) {
+    const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
+    const float x = slot[e];
+    const u64 key = cand_key(x, (uint32_t)(tok_tile + e));
+    bool ok = ((mm >> i) & 1u) && x >= w.thr_f && key > w.thr_key;
+    unsigned mk = __ballot_sync(FULL, ok);
+    if (mk == 0u) continue;
+    if (w.cnt + __popc(mk) > XS_BUF) {
+      cut_back(buf, ke, w, lane);
+      ok = ok && x >= w.thr_f && key > w.thr_key;
+      mk = __ballot_sync(FULL, ok);
+    }
+    if (ok) buf[w.cnt + __popc(mk & ((1u << lane) - 1u))] = key;
+    w.cnt += __popc(mk);
+    __syncwarp();
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Selection phase
+// ---------------------------------------------------------------------------------------
+// Shared-memory carve-up of the selection phase (it reuses the streaming ring).
 struct TailSmem {
-  u64 *stage;        // [EXP_WARPS][32 k + FX_SURV]  chunk lists of the row a warp is merging, survivors
+  u64 *stage;        // [EXP_WARPS][FX_MAX_SPLITS k + FX_SURV + k]  chunk lists of the row a warp is merging, survivors, result
   u64 *row_keys;     // [N-1][k]               per-row top-k keys, descending
   double *score;     // [N-1][k]               log p(u) of each pooled candidate
-  double *row_t;     // [N-1]                  sum of exponentials relative to row_m
-  double *row_ps;    // [N-1]                  log p(v) of the row's parent
   u64 *row_mask;     // [N-1][W]               ancestor mask of the row's parent
-  float *row_m;      // [N-1]
   int *row_cnt, *row_off;   // [N-1]
   unsigned char *state;     // [N-1][k]        bit0 eligible, bit2 selected
 };
 
-// Leaves a frontier row's maximum m and sum of exponentials t for the scoring phase, which takes
-// the logarithm once per candidate, in parallel (one thread taking it here would hold up its whole
-// warp).  m + log t is a finite number exactly when m is finite and 0 < t < inf; anything else
-// (a NaN or +inf logit, a row of -inf only) flags the sequence.
-__device__ __forceinline__ void finish_row(const FusedArgs &a, const TailSmem &sm, int j, float m, double t,
-                                           int *s_bad) {
-  if (!(t > 0.0) || !(t < CUDART_INF) || !(m < CUDART_INF_F) || !(m > -CUDART_INF_F)) {
-    *s_bad = 1;
-    atomicOr(a.status, STATUS_NONFINITE);
-  }
-  sm.row_m[j] = m;
-  sm.row_t[j] = t;
-  sm.row_cnt[j] = 0;
-}
+__device__ inline int stage_words(int k) { return FX_MAX_SPLITS * k + FX_SURV + k; }
 
-__device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int lo, int row0, int F, int S,
-                            u64 *s_anchor, int *s_cnt, int *s_bad) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int k = a.k, ks = a.key_stride;
-  const int n = a.t.n_nodes[b];
-  const int R = a.N - n;
-  const int ke = min(k, R);                 // a parent can place at most R children
-  const size_t nb = (size_t)b * a.N;
-
-  // ---- per row: chunk normalisers -> (max, sum); chunk lists -> the row's k best keys.
-  // One warp per row, one lane per chunk (S <= 32). ----
-  const int stage_words = 32 * k + FX_SURV;
-  // Many rows means few chunks per row (their product is bounded by the grid): then all rows
-  // are merged at once, one thread per key, instead of a row at a time per warp.  Up to two
-  // rounds of the warp-per-row merge measured faster than the flat one (10 rows x 8 chunks:
-  // 4 us per layer), hence the bound on F.
-  const bool flat = S > 1 && S <= 8 && F > 2 * EXP_WARPS && F * S * k <= EXP_WARPS * stage_words;
-  if (flat) {
-    const size_t item0 = (size_t)row0 * S;
-    u64 *st = sm.stage;                           // st[(j * S + c) * k + i]
-    const int nkeys = F * S * k;
-    // The compiler cannot move a global load above a store through a shared-memory pointer it
-    // cannot tell apart, so every round of loads goes to registers before anything is stored:
-    // one trip to L2 per round instead of one per load.
-    auto key_at = [&](int idx) {
-      const int jc = idx / k, i = idx - jc * k;
-      return __ldcg(a.part_keys + (item0 + jc) * ks + i);
-    };
-    const u64 key_first = tid < nkeys ? key_at(tid) : 0ull;
-    if (tid < F) {
-      const int j = tid;
-      float2 ms[8];
+// One warp merges the S chunk results of the frontier row of tree node `node` (index into the
+// [B, N] arrays).  Afterwards lane i < k holds the row's i-th best key and its score
+// log p(v) + (z - lse) (Eq. 2-3; -inf for an empty slot or one past the ke children the budget
+// still allows), and lane w < W word w of the parent's ancestor mask.  Returns false, for the whole warp, when the row's
+// normaliser is not a positive finite number (a NaN or +inf logit, a row of -inf only).
+__device__ __forceinline__ bool merge_row(const FusedArgs &a, size_t item0, int S, int k, int ke, size_t node, u64 *st,
+                                          u64 &out_key, double &out_score, u64 &out_mask) {
+  const int lane = threadIdx.x & 31;
+  const int ks = a.key_stride;
+  u64 *sv = st + FX_MAX_SPLITS * k;              // keys that reach the bound
+  u64 *rk = sv + FX_SURV;                        // the row's k best keys
+  // Everything this row needs from global memory goes to registers before the first store (a
+  // load cannot pass a store through a pointer the compiler cannot tell apart): one trip to L2
+  // for the row, not one per load.
+  const float2 ms = (lane < S) ? __ldcg(a.part_ms + item0 + lane) : make_float2(-CUDART_INF_F, 0.f);
+  const double ps = a.t.score[node];                                    // log p(v) of the row's parent
+  out_mask = lane < a.W ? a.t.mask[node * a.W + lane] : 0ull;           // and its ancestor-mask row
+  if (S == 1) {
+    const u64 key = lane < k ? __ldcg(a.part_keys + item0 * ks + lane) : 0ull;
+    if (lane < k) rk[lane] = key;
+  } else {
+    const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(a.part_keys + (item0 + min(lane, S - 1)) * ks);
+    for (int i0 = 0; i0 < k; i0 += 16) {         // slots k..ks-1 of a list always hold zero
+      ulonglong2 x[8];
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
-        ms[c] = c < S ? __ldcg(a.part_ms + item0 + (size_t)j * S + c) : make_float2(-CUDART_INF_F, 0.f);
-      const double ps = a.t.score[nb + lo + j];
-      u64 mk[4];
+      for (int u = 0; u < 8; ++u)
+        x[u] = (lane < S && i0 + 2 * u < k) ? __ldcg(src + i0 / 2 + u) : make_ulonglong2(0ull, 0ull);
 #pragma unroll
-      for (int w = 0; w < 4; ++w) mk[w] = w < a.W ? a.t.mask[(nb + lo + j) * a.W + w] : 0ull;
-      float mx = -CUDART_INF_F;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) mx = fmaxf(mx, ms[c].x);
-      double t = 0.0;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        if (ms[c].y != ms[c].y) t += (double)ms[c].y;                     // NaN or +inf logit in the chunk
-        else if (ms[c].x > -CUDART_INF_F) t += (double)ms[c].y * (double)exp2f((ms[c].x - mx) * LOG2E_F);
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + 2 * u;
+        if (lane < S && i < k) st[i * FX_MAX_SPLITS + lane] = x[u].x;
+        if (lane < S && i + 1 < k) st[(i + 1) * FX_MAX_SPLITS + lane] = x[u].y;
       }
-      sm.row_ps[j] = ps;
-#pragma unroll
-      for (int w = 0; w < 4; ++w)
-        if (w < a.W) sm.row_mask[j * a.W + w] = mk[w];
-      for (int w = 4; w < a.W; ++w) sm.row_mask[j * a.W + w] = a.t.mask[(nb + lo + j) * a.W + w];
-      finish_row(a, sm, j, mx, t, s_bad);
-    }
-    if (tid < nkeys) st[tid] = key_first;
-    for (int idx = tid + EXP_THREADS; idx < nkeys; idx += 2 * EXP_THREADS) {
-      const u64 k0 = key_at(idx);
-      const u64 k1 = idx + EXP_THREADS < nkeys ? key_at(idx + EXP_THREADS) : 0ull;
-      st[idx] = k0;
-      if (idx + EXP_THREADS < nkeys) st[idx + EXP_THREADS] = k1;
-    }
-    for (int idx = tid; idx < F * k; idx += EXP_THREADS) sm.row_keys[idx] = 0ull;
-    __syncthreads();
-    // a key's rank in its row: its place in its own list plus, for every other chunk of the
-    // row, how many of that chunk's keys beat it (keys are unique; lists are descending)
-    for (int idx = tid; idx < nkeys; idx += EXP_THREADS) {
-      const u64 key = st[idx];
-      if (key == 0ull) continue;
-      const int jc = idx / k, i = idx - jc * k;
-      const int j = jc / S, c = jc - j * S;
-      int rank = i;
-      for (int o = 0; o < S; ++o) {
-        if (o == c) continue;
-        const u64 *lst = st + (size_t)(j * S + o) * k;
-        int l = 0, h = k;
-        while (l < h) {
-          const int mid = (l + h) >> 1;
-          if (lst[mid] > key) l = mid + 1; else h = mid;
-        }
-        rank += l;
-      }
-      if (rank < k) sm.row_keys[(size_t)j * k + rank] = key;
     }
   }
-  for (int j = flat ? F : warp; j < F; j += EXP_WARPS) {
-    const size_t item0 = (size_t)(row0 + j) * S;
-    u64 *st = sm.stage + warp * stage_words;       // st[i * 32 + c] = i-th best key of chunk c
-    u64 *sv = st + 32 * k;                         // keys that reach the bound
-    u64 *rk = sm.row_keys + (size_t)j * k;
-    // Everything this row needs from global memory goes to registers before the first store
-    // (a load cannot pass a store through a pointer the compiler cannot tell apart): one trip
-    // to L2 for the row, not one per load.
-    const float2 ms = (lane < S) ? __ldcg(a.part_ms + item0 + lane) : make_float2(-CUDART_INF_F, 0.f);
-    const double ps = lane == 0 ? a.t.score[nb + lo + j] : 0.0;
-    const u64 pmask = lane < a.W ? a.t.mask[(nb + lo + j) * a.W + lane] : 0ull;
-    if (S == 1) {
-      const u64 key = lane < k ? __ldcg(a.part_keys + item0 * ks + lane) : 0ull;
-      if (lane < k) rk[lane] = key;
-    } else {
-      const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(a.part_keys + (item0 + min(lane, S - 1)) * ks);
-      for (int i0 = 0; i0 < k; i0 += 16) {         // slots k..ks-1 of a list always hold zero
-        ulonglong2 x[8];
+  float mx = ms.x;
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          x[u] = (lane < S && i0 + 2 * u < k) ? __ldcg(src + i0 / 2 + u) : make_ulonglong2(0ull, 0ull);
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+  double t = 0.0;
+  if (ms.y != ms.y) t = (double)ms.y;                                   // NaN or +inf logit in the chunk
+  else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = i0 + 2 * u;
-          if (lane < S && i < k) st[i * 32 + lane] = x[u].x;
-          if (lane < S && i + 1 < k) st[(i + 1) * 32 + lane] = x[u].y;
-        }
-      }
-    }
-    if (lane == 0) sm.row_ps[j] = ps;
-    if (lane < a.W) sm.row_mask[j * a.W + lane] = pmask;
+  for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
+  const bool finite = (t > 0.0) && (t < CUDART_INF) && (mx < CUDART_INF_F) && (mx > -CUDART_INF_F);
 
-    float mx = ms.x;
-#pragma unroll
-    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
-    double t = 0.0;
-    if (ms.y != ms.y) t = (double)ms.y;                                   // NaN or +inf logit in the chunk
-    else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
-#pragma unroll
-    for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
-    if (lane == 0) finish_row(a, sm, j, mx, t, s_bad);
-    if (S == 1) continue;
-
+  if (S > 1) {
     if (lane < k) rk[lane] = 0ull;
-    // Two lower bounds of the row's k-th best key: the best k-th key of any one chunk, and the
-    // k-th best of the chunk heads (k different chunks each hold a key at least that large).
+    __syncwarp();
+    // Two lower bounds of the row's ke-th best key (chunk lists hold ke keys at most): the best
+    // ke-th key of any one chunk, and the ke-th best of the chunk heads (ke different chunks each
+    // hold a key at least that large).
     const u64 head = lane < S ? st[lane] : 0ull;
-    u64 tau = lane < S ? st[(k - 1) * 32 + lane] : 0ull;
-    if (S >= k) {
+    u64 tau = lane < S ? st[(ke - 1) * FX_MAX_SPLITS + lane] : 0ull;
+    if (S >= ke) {
       int cnt = 0;
 #pragma unroll 8
       for (int o = 0; o < 32; ++o) cnt += (shfl_u64(head, o) > head) ? 1 : 0;
-      if (cnt == k - 1) tau = umax64(tau, head);
+      if (cnt == ke - 1) tau = umax64(tau, head);
     }
     tau = warp_max_u64(tau);
     // keys that reach the bound: lists are sorted, so the scan over list positions stops at the
     // first position where no chunk has one
     int ns = 0;
-    for (int i = 0; i < k; ++i) {
-      const u64 key = lane < S ? st[i * 32 + lane] : 0ull;
+    for (int i = 0; i < ke; ++i) {
+      const u64 key = lane < S ? st[i * FX_MAX_SPLITS + lane] : 0ull;
       const bool ok = key != 0ull && key >= tau;
       const unsigned mk = __ballot_sync(FULL, ok);
       if (mk == 0u) break;
@@ -487,42 +556,42 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int l
         const u64 key = sv[i];
         int r = 0;
         for (int o = 0; o < ns; ++o) r += (sv[o] > key) ? 1 : 0;
-        if (r < k) rk[r] = key;
+        if (r < ke) rk[r] = key;
       }
     } else {
-      // many keys at the bound (equal logits): pop the largest head k times
+      // many keys at the bound (equal logits): pop the largest head ke times
       int p = 0;
-      for (int r = 0; r < k; ++r) {
-        const u64 cand = (lane < S && p < k) ? st[p * 32 + lane] : 0ull;
+      for (int r = 0; r < ke; ++r) {
+        const u64 cand = (lane < S && p < ke) ? st[p * FX_MAX_SPLITS + lane] : 0ull;
         const u64 best = warp_max_u64(cand);
         if (best == 0ull) break;
         if (cand == best) ++p;
         if (lane == 0) rk[r] = best;
       }
     }
-    __syncwarp();
   }
-  __syncthreads();
-
-  if (*s_bad) {            // a frontier row was not finite: this sequence adds nothing
-    if (tid == 0) a.t.layer_off[b * a.lo_stride + a.d + 2] = n;
-    return;
+  __syncwarp();
+  out_key = lane < k ? rk[lane] : 0ull;
+  out_score = -CUDART_INF;
+  if (finite && lane < ke && out_key != 0ull) {
+    const double s = ps + ((double)key_logit(out_key) - ((double)mx + log(t)));
+    if (s == s && s > -CUDART_INF) out_score = s;
   }
+  __syncwarp();
+  return finite;
+}
 
-  // ---- pool: log p(u) = log p(v) + (z_w - lse_v)   (Eq. 2-3) ----
+// Gate, budget truncation and append for one sequence, from the pooled candidates in shared
+// memory (sm.row_keys / sm.score: F rows of k, each row descending; sm.row_mask: the parents'
+// mask rows).  n is the tree's size before the layer.
+__device__ void select_and_append(const FusedArgs &a, const TailSmem &sm, int b, int lo, int F, int n,
+                                  u64 *s_anchor, int *s_cnt) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k = a.k;
+  const int R = a.N - n;
+  const int ke = min(k, R);                 // a parent can place at most R children
+  const size_t nb = (size_t)b * a.N;
   const int C = F * k;
-  for (int c = tid; c < C; c += EXP_THREADS) {
-    const int j = c / k, i = c - j * k;
-    const u64 key = sm.row_keys[c];
-    double s = -CUDART_INF;
-    if (i < ke && key != 0ull) s = sm.row_ps[j] + ((double)key_logit(key) - ((double)sm.row_m[j] + log(sm.row_t[j])));
-    const bool ok = (s > -CUDART_INF) && (s == s);
-    if (!ok) s = -CUDART_INF;
-    sm.score[c] = s;
-    sm.state[c] = ok ? 1 : 0;
-    if (ok && i == 0) atomicMax(s_anchor, f64_ord(s));        // rows are sorted: heads carry the maxima
-  }
-  __syncthreads();
 
   // ---- eligibility: Top-K layers take every candidate, gated layers Eq. 4 ----
   const bool init = a.d < a.init_layers;
@@ -530,11 +599,13 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int l
   if (!init && *s_anchor != 0ull) thr = a.log_mu + f64_unord(*s_anchor);
   int local = 0;
   for (int c = tid; c < C; c += EXP_THREADS) {
-    unsigned char stt = sm.state[c];
-    if (stt && !init && !(sm.score[c] >= thr)) stt = 0;
+    const double s = sm.score[c];
+    unsigned char stt = (s > -CUDART_INF) ? 1 : 0;
+    if (stt && !init && !(s >= thr)) stt = 0;
     sm.state[c] = stt;
     local += stt;
   }
+  for (int j = tid; j < F; j += EXP_THREADS) sm.row_cnt[j] = 0;
 #pragma unroll
   for (int o = 16; o; o >>= 1) local += __shfl_xor_sync(FULL, local, o);
   if (lane == 0 && local) atomicAdd(s_cnt, local);
@@ -615,178 +686,46 @@ __device__ void select_tail(const FusedArgs &a, const TailSmem &sm, int b, int l
   }
 }
 
-// Per-warp state of the streamed top-k: a sorted list across the lanes (once something was
-// folded), a queue in shared memory, and the threshold an element has to reach.
-struct WarpTopk {
-  u64 list;
-  bool folded, first;
-  int qn;
-  float thr0, thr_f;
-};
-
-// One tile (16 elements per thread, already in registers) through the warp's threshold queue.
-// bm is the thread's maximum over the tile.
-__device__ __forceinline__ void topk_tile(const float (&v)[EXP_UNROLL][EXP_VEC], float bm, int base, int end, int k,
-                                          u64 *queue, int *qcnt, unsigned *thr_cta, WarpTopk &w) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  const bool was_first = w.first;
-  if (w.first) {
-    w.first = false;
-    // k lane maxima are k distinct elements, so the k-th largest lane maximum is a lower
-    // bound of this warp's k-th largest element: nothing below it needs to be looked at.
-    int rank = 0;
-#pragma unroll
-    for (int l = 0; l < 32; ++l) {
-      const float o = __shfl_sync(FULL, bm, l);
-      rank += (o > bm) || (o == bm && l < lane);
-    }
-    const unsigned pick = __ballot_sync(FULL, rank == k - 1);
-    if (pick) w.thr0 = __shfl_sync(FULL, bm, __ffs(pick) - 1);
-    w.thr_f = w.thr0;
-  }
-  // A thread holds something at or above the threshold iff its maximum over the tile is: one
-  // compare per tile.  The threshold is shared by the CTA's warps: whenever a warp sorts its
-  // keys, its k-th best key is a lower bound of the chunk's k-th largest element for everybody.
-  {
-    const unsigned shared_thr = *thr_cta;
-    if (shared_thr) w.thr_f = fmaxf(w.thr_f, f32_unord(shared_thr));
-  }
-  const bool hit = bm >= w.thr_f;
-  const unsigned hm = __ballot_sync(FULL, hit);
-  if (hm == 0u) return;
-  if (__popc(hm) <= 6) {
-    // a few lanes hold everything that reaches the threshold: only they look at their elements
-    // (at most 6 x 16 new keys; fewer than 32 were waiting)
-    if (lane == 0) *qcnt = w.qn;
-    __syncwarp();
-    if (hit) {
-#pragma unroll
-      for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-        for (int e = 0; e < EXP_VEC; ++e) {
-          const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-          if (v[u][e] >= w.thr_f && tok < end) queue[atomicAdd(qcnt, 1)] = cand_key(v[u][e], (uint32_t)tok);
-        }
-    }
-    __syncwarp();
-    w.qn = *qcnt;
-    while (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
-    return;
-  }
-  int mine = 0;
-#pragma unroll
-  for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-    for (int e = 0; e < EXP_VEC; ++e)
-      mine += (v[u][e] >= w.thr_f && base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e < end) ? 1 : 0;
-  if (!__any_sync(FULL, mine > 0)) return;
-  int inc = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(FULL, inc, o);
-    if (lane >= o) inc += t;
-  }
-  const int total = __shfl_sync(FULL, inc, 31);
-  if (total <= 32) {
-    int pos = w.qn + inc - mine;
-#pragma unroll
-    for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-      for (int e = 0; e < EXP_VEC; ++e) {
-        const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-        if (v[u][e] >= w.thr_f && tok < end) queue[pos++] = cand_key(v[u][e], (uint32_t)tok);
-      }
-    w.qn += total;
-    __syncwarp();
-    if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
-    else if (was_first && w.qn >= k) {
-      // the first tile's bound is loose: sort what it let through so that the k-th best key of
-      // this tile becomes the threshold for the next ones
-      flush_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane);
-      w.folded = true;
-      publish_thr(thr_cta, w.thr_f, lane);
-    }
-  } else {
-    // many elements at or above the threshold (equal logits, or a cold threshold): one
-    // register slot at a time, folding whenever 32 keys are waiting
-#pragma unroll
-    for (int u = 0; u < EXP_UNROLL; ++u) {
-#pragma unroll
-      for (int e = 0; e < EXP_VEC; ++e) {
-        const int tok = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e;
-        const bool ok = v[u][e] >= w.thr_f && tok < end;
-        const unsigned mk = __ballot_sync(FULL, ok);
-        if (mk == 0u) continue;
-        if (ok) queue[w.qn + __popc(mk & ((1u << lane) - 1u))] = cand_key(v[u][e], (uint32_t)tok);
-        w.qn += __popc(mk);
-        __syncwarp();
-        if (w.qn >= 32) { fold_queue(w.list, w.qn, w.thr_f, queue, w.thr0, k, lane); w.folded = true; publish_thr(thr_cta, w.thr_f, lane); }
-      }
-    }
-  }
-}
-
-// The warp's best keys (list and queue) -> the CTA pool.
-__device__ __forceinline__ void pool_from_warp(WarpTopk &w, u64 *queue, u64 *s_pool, int *s_pool_n, int k) {
-  const int lane = threadIdx.x & 31;
-  int cnt_w = w.qn;
-  if (w.folded) {
-    if (w.qn > 0) w.list = warp_merge_desc(w.list, lane < w.qn ? queue[lane] : 0ull, lane);
-    cnt_w = __popc(__ballot_sync(FULL, lane < k && w.list != 0ull));
-  }
-  int pos = 0;
-  if (lane == 0) pos = atomicAdd(s_pool_n, cnt_w);
-  pos = __shfl_sync(FULL, pos, 0);
-  if (lane < cnt_w) s_pool[pos + lane] = w.folded ? w.list : queue[lane];
-}
-
-__device__ __forceinline__ void load_tile(float (&v)[EXP_UNROLL][EXP_VEC], const float *rowp, int base, int end) {
-  const int tid = threadIdx.x;
-#pragma unroll
-  for (int u = 0; u < EXP_UNROLL; ++u) {
-    const int idx = base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
-    if (idx + EXP_VEC <= end) {
-      const float4 x = __ldcs(reinterpret_cast<const float4 *>(rowp + idx));
-      v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-    } else {
-#pragma unroll
-      for (int e = 0; e < EXP_VEC; ++e) v[u][e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
-    }
-  }
-}
-
 __global__ void __launch_bounds__(EXP_THREADS, 3)
 expand_fused_kernel(FusedArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  __shared__ u64 s_queue[EXP_WARPS][FX_QCAP];       // per-warp queues of keys above the threshold
-  __shared__ u64 s_pool[FX_POOL];                   // the chunk's candidates, all warps
+  __shared__ u64 s_buf[EXP_WARPS][XS_BUF];          // per-warp buffers of keys that reached the threshold
+  __shared__ u64 s_pool[XS_POOL];                   // the chunk's candidates, all warps
   __shared__ int s_base[MAX_BATCH + 1];
   __shared__ int s_warp[EXP_WARPS];
   __shared__ float s_m[EXP_WARPS], s_s[EXP_WARPS];
-  __shared__ __align__(8) unsigned long long s_ring_bar[FX_RING];   // "tile landed" barriers
-  __shared__ unsigned s_thr_cta;                    // ordered bits of the CTA-wide threshold (0: none yet)
-  __shared__ int s_qn[EXP_WARPS];                   // queue fill, when lanes append on their own
-  __shared__ float s_gmax[32];                      // maxima of lane groups (single-tile chunks)
+  __shared__ __align__(8) u64 s_bar[EXP_WARPS][XS_RING];   // "tile landed" barriers, per warp
+  __shared__ float s_wtop[EXP_WARPS];               // each warp's ceil(k/8)-th largest lane maximum
+  __shared__ float s_wmax[EXP_WARPS];               // each warp's largest
   __shared__ u64 s_anchor;
-  __shared__ int s_pool_n, s_last, s_cnt, s_bad;
+  __shared__ int s_pool_n, s_last, s_last_seq, s_ecnt, s_bad, s_abort;
 
-  pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = a.k;
+  if (lane == 0) {
+    for (int i = 0; i < XS_RING; ++i) ring_bar_init(smem_addr(&s_bar[warp][i]));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_wtop[warp] = -CUDART_INF_F;
+    s_wmax[warp] = -CUDART_INF_F;
+  }
+  if (tid == 0) {
+    s_pool_n = 0; s_abort = 0;
+    s_anchor = 0ull; s_ecnt = 0; s_bad = 0;
+  }
+  pdl_enter();
 
-  // ---- frontier geometry ----
+  // ---- frontier geometry (from layer_off[d], layer_off[d + 1]: never written by this launch) ----
   Frontier fr;
   fr.in_regs = a.B <= 32;
   fr.s_base = s_base;
   fr.base_l = fr.f_l = fr.lo_l = 0;
   if (fr.in_regs) {
     if (lane < a.B) {
-      const int nn = a.t.n_nodes[lane];
       fr.lo_l = a.t.layer_off[lane * a.lo_stride + a.d];
       const int hi = a.t.layer_off[lane * a.lo_stride + a.d + 1];
-      fr.f_l = nn < a.N ? max(hi - fr.lo_l, 0) : 0;
+      fr.f_l = hi < a.N ? max(hi - fr.lo_l, 0) : 0;
       if (fr.f_l == 0 && blockIdx.x == 0 && warp == 0)        // nothing to expand: close the layer
-        a.t.layer_off[lane * a.lo_stride + a.d + 2] = nn;
+        a.t.layer_off[lane * a.lo_stride + a.d + 2] = hi;
     }
     int inc = fr.f_l;
 #pragma unroll
@@ -801,23 +740,27 @@ expand_fused_kernel(FusedArgs a) {
     fr.total = s_base[a.B];
     if (blockIdx.x == 0)
       for (int b = tid; b < a.B; b += EXP_THREADS)
-        if (s_base[b + 1] == s_base[b]) a.t.layer_off[b * a.lo_stride + a.d + 2] = a.t.n_nodes[b];
+        if (s_base[b + 1] == s_base[b])
+          a.t.layer_off[b * a.lo_stride + a.d + 2] = a.t.layer_off[b * a.lo_stride + a.d + 1];
   }
-  if (tid == 0) {
-    s_pool_n = 0;
-    s_thr_cta = 0u;
-    for (int i = 0; i < FX_RING; ++i) ring_bar_init(smem_addr(&s_ring_bar[i]));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  unsigned ring_tiles = 0;         // tiles this CTA has taken from the ring so far (all threads agree)
-  const LayerGeom g = balanced_geom(fr.total, a.V, a.target_items, a.max_splits, a.items_cap);
-  const int n_items = fr.total * g.splits;
-  // lanes per group whose maxima bound the k-th largest element of a single-tile chunk
-  const int grp = k <= 8 ? 32 : (k <= 16 ? 16 : 8);
+  const SpanGeom g = span_geom(fr.total, a.V, (int)gridDim.x, a.max_split);
+  const unsigned long long line_end = (unsigned long long)fr.total * g.pitch;
+  const bool gated = a.d >= a.init_layers;
+  const float ln_mu = (float)a.log_mu;
+  unsigned wt = 0;                 // tiles this warp has taken from its ring so far
+  float *ring = reinterpret_cast<float *>(smem_raw) + warp * (XS_RING * XS_WTILE);
+  u64 *buf = s_buf[warp];
   __syncthreads();
 
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int row = item / g.splits, chunk = item - row * g.splits;
+  unsigned long long pos = (unsigned long long)blockIdx.x * g.span;
+  const unsigned long long span_end = min(line_end, pos + g.span);
+  int row = pos < span_end ? (int)div_u64(pos, g.pitch) : 0;
+  int start = pos < span_end ? (int)(pos - (unsigned long long)row * g.pitch) : 0;
+  for (; pos < span_end; ++row, start = 0) {
+    // ---- one chunk: elements [start, start + len) of packed row `row` ----
+    const int len = (int)min((unsigned long long)(g.pitch - (unsigned)start), span_end - pos);
+    pos += (unsigned)len;
+    const int item = (int)blockIdx.x + row;
     const RowLoc rl = locate_row(a, fr, row);
     int rsel = (a.layout == TALON_ROWS_BY_NODE) ? rl.node : rl.j;
     if (rsel >= a.rows_per_seq) {               // caller reserved too few rows: stay in bounds, report
@@ -825,163 +768,143 @@ expand_fused_kernel(FusedArgs a) {
       if (tid == 0) atomicOr(a.status, STATUS_CAPACITY);
     }
     const float *rowp = a.logits + ((int64_t)rl.b * a.rows_per_seq + rsel) * a.row_stride;
-    const int start = chunk * g.chunk_len;
-    const int end = min(a.V, start + g.chunk_len);
-    u64 *queue = s_queue[warp];
-    float wm, ws;                    // this warp's maximum and sum of exponentials relative to it
+    const int end = min(a.V, start + len);        // (an empty chunk past the row's end still reports in)
+    const int lo = rl.node - rl.j;               // first frontier node of the sequence
+    const int n_before = lo + rl.F;              // the tree's size before this layer
+    const int ke = min(k, a.N - n_before);       // a parent can place at most N - |T| children
+    const int share_pos = (ke + EXP_WARPS - 1) / EXP_WARPS - 1;
 
-    if (end - start <= EXP_TILE) {
-      // ---- the whole chunk in registers ----
-      float v[EXP_UNROLL][EXP_VEC];
-      load_tile(v, rowp, start, end);
-      float bm = -CUDART_INF_F;
-#pragma unroll
-      for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-        for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
-      float g8 = bm;
-#pragma unroll
-      for (int o = 1; o < 8; o <<= 1) g8 = fmaxf(g8, __shfl_xor_sync(FULL, g8, o));
-      const float g16 = fmaxf(g8, __shfl_xor_sync(FULL, g8, 8));
-      wm = fmaxf(g16, __shfl_xor_sync(FULL, g16, 16));
-      float acc = 0.f;
-      if (wm > -CUDART_INF_F) {
-#pragma unroll
-        for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) acc += fast_exp2(fmaf(v[u][e], LOG2E_F, -wm * LOG2E_F));
+    // ---- this warp's slice of the chunk ----
+    // (a short chunk goes to fewer warps, a full tile each: thresholds need elements to work with)
+    const int wlen = max(XS_WTILE, ((end - start + 4 * EXP_WARPS - 1) / (4 * EXP_WARPS)) * 4);
+    const int ws = start + warp * wlen;
+    const int we = min(end, ws + wlen);
+    const int nt = ws < we ? (we - ws + XS_WTILE - 1) / XS_WTILE : 0;
+    auto issue = [&](int t, unsigned slot_index) {
+      const int base = ws + t * XS_WTILE;
+      const int n = min(XS_WTILE, we - base);
+      const unsigned sl = slot_index % XS_RING;
+      // whole 16-byte units: the last one of a row may reach into the row's stride padding
+      ring_issue(smem_addr(ring + sl * XS_WTILE), rowp + base, (uint32_t)(((n * 4) + 15) & ~15),
+                 smem_addr(&s_bar[warp][sl]));
+    };
+    if (lane == 0)
+      for (int t = 0; t < nt && t < XS_RING; ++t) issue(t, wt + t);
+    WarpStream w;
+    w.m_t = -CUDART_INF_F; w.s_t = 0.f;
+    w.thr_f = -CUDART_MAX_NORMAL_F;              // -inf never competes (probability zero)
+    w.thr_key = 0ull;
+    w.cnt = 0;
+    bool refreshed = false;
+    for (int t = 0; t < nt; ++t) {
+      const int base = ws + t * XS_WTILE;
+      const unsigned sl = wt % XS_RING;
+      if (!ring_wait(smem_addr(&s_bar[warp][sl]), (wt / XS_RING) & 1u)) {
+        // The copy did not land in time: the launch is reported as timed out (the tree arrays are
+        // undefined from here on) and the CTA leaves at the end of this chunk.  The copy gets one
+        // more bounded wait so that it does not land in memory the CTA has already given back.
+        if (lane == 0) { atomicOr(a.status, STATUS_TIMEOUT); s_abort = 1; }
+        ring_wait(smem_addr(&s_bar[warp][sl]), (wt / XS_RING) & 1u);
       }
-      ws = acc;
+      float v[16];
 #pragma unroll
-      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
-      if ((lane & (grp - 1)) == 0) s_gmax[(tid / grp)] = grp == 32 ? wm : (grp == 16 ? g16 : g8);
-      if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
-      __syncthreads();
-      // the smallest group maximum: at least 256/grp >= k elements of the chunk reach it
-      float tau = lane < EXP_THREADS / grp ? s_gmax[lane] : CUDART_INF_F;
-#pragma unroll
-      for (int o = 16; o; o >>= 1) tau = fminf(tau, __shfl_xor_sync(FULL, tau, o));
-      // Only a thread whose own maximum reaches the bound holds candidates (about 8 H(8) = 22 of
-      // the 256 do): those append to the CTA's pool themselves.  -inf never competes (probability
-      // zero, and it is what the slots past `end` hold), so the bound is kept finite.
-      const float tau_f = fmaxf(tau, -CUDART_MAX_NORMAL_F);
-      if (bm >= tau_f) {
-#pragma unroll
-        for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e)
-            if (v[u][e] >= tau_f) {
-              const int pos = atomicAdd(&s_pool_n, 1);
-              if (pos < FX_POOL)
-                s_pool[pos] = cand_key(v[u][e], (uint32_t)(start + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e));
-            }
+      for (int u = 0; u < 4; ++u) {
+        const float4 x = *reinterpret_cast<const float4 *>(ring + sl * XS_WTILE + u * 128 + lane * 4);
+        v[4 * u + 0] = x.x; v[4 * u + 1] = x.y; v[4 * u + 2] = x.z; v[4 * u + 3] = x.w;
       }
-      __syncthreads();
-      if (s_pool_n > FX_POOL) {
-        // too many elements at the bound (equal logits, masked vocabulary, a tiny chunk): take
-        // the per-warp queue route on the same registers
-        __syncthreads();
-        if (tid == 0) s_pool_n = 0;
-        __syncthreads();
-        WarpTopk w;
-        w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
-        w.thr0 = w.thr_f = -CUDART_INF_F;
-        topk_tile(v, bm, start, end, k, queue, &s_qn[warp], &s_thr_cta, w);
-        pool_from_warp(w, queue, s_pool, &s_pool_n, k);
-        __syncthreads();
+      if (base + XS_WTILE > we) {             // the slice's last, partial tile: nothing past `we` counts
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (base + (i >> 2) * 128 + lane * 4 + (i & 3) >= we) v[i] = -CUDART_INF_F;
       }
-    } else {
-      // ---- a longer chunk, streamed tile by tile ----
-      float m_t = -CUDART_INF_F, s_t = 0.f;
-      WarpTopk w;
-      w.list = 0ull; w.folded = false; w.first = true; w.qn = 0;
-      w.thr0 = w.thr_f = -CUDART_INF_F;
-      const int nt = (end - start + EXP_TILE - 1) / EXP_TILE;
-      float *ring = reinterpret_cast<float *>(smem_raw);        // FX_RING tiles; the selection phase reuses it
-      auto issue = [&](int t, unsigned slot_index) {
-        const int base = start + t * EXP_TILE;
-        const int n = min(EXP_TILE, end - base);
-        const unsigned st = slot_index % FX_RING;
-        // whole 16-byte units: the last one may reach into the row's stride padding
-        ring_issue(smem_addr(ring + st * EXP_TILE), rowp + base, (uint32_t)(((n * 4) + 15) & ~15),
-                   smem_addr(&s_ring_bar[st]));
-      };
-      if (tid == 0)
-        for (int t = 0; t < nt && t < FX_RING; ++t) issue(t, ring_tiles + t);
-      for (int t = 0; t < nt; ++t) {
-        const int base = start + t * EXP_TILE;
-        const unsigned st = ring_tiles % FX_RING;
-        const bool landed = ring_wait(smem_addr(&s_ring_bar[st]), (ring_tiles / FX_RING) & 1u);
-        float v[EXP_UNROLL][EXP_VEC];
-#pragma unroll
-        for (int u = 0; u < EXP_UNROLL; ++u) {
-          const int off = u * EXP_CHUNK_ALIGN + tid * EXP_VEC;
-          const float4 x = *reinterpret_cast<const float4 *>(ring + st * EXP_TILE + off);
-          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-        }
-        if (base + EXP_TILE > end) {          // the chunk's last, partial tile: nothing past `end` counts
-#pragma unroll
-          for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-            for (int e = 0; e < EXP_VEC; ++e)
-              if (base + u * EXP_CHUNK_ALIGN + tid * EXP_VEC + e >= end) v[u][e] = -CUDART_INF_F;
-        }
-        // every thread has its copy of the tile: the slot can take the tile FX_RING ahead
-        if (!__syncthreads_and(landed)) {
-          if (tid == 0) atomicOr(a.status, STATUS_TIMEOUT);
-          return;
-        }
-        if (tid == 0 && t + FX_RING < nt) {
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          issue(t + FX_RING, ring_tiles + FX_RING);
-        }
-        ++ring_tiles;
-        float bm = -CUDART_INF_F;
-#pragma unroll
-        for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-          for (int e = 0; e < EXP_VEC; ++e) bm = fmaxf(bm, v[u][e]);
-        // running softmax normaliser of this thread's elements
-        if (bm > m_t) {
-          s_t *= fast_exp2((m_t - bm) * LOG2E_F);
-          m_t = bm;
-        }
-        if (m_t > -CUDART_INF_F) {
-          // exp(v - m) = 2^(v * log2e - m * log2e); an infinite m (a +inf logit) must give NaN
-          const float c = -m_t * LOG2E_F;
-          float acc = 0.f;
-#pragma unroll
-          for (int u = 0; u < EXP_UNROLL; ++u)
-#pragma unroll
-            for (int e = 0; e < EXP_VEC; ++e) acc += fast_exp2(fmaf(v[u][e], LOG2E_F, c));
-          s_t += acc;
-        }
-        topk_tile(v, bm, base, end, k, queue, &s_qn[warp], &s_thr_cta, w);
+      ++wt;
+      float bm = max3(max3(v[0], v[1], v[2]), max3(v[3], v[4], v[5]), max3(v[6], v[7], v[8]));
+      bm = max3(bm, max3(v[9], v[10], v[11]), max3(v[12], v[13], v[14]));
+      bm = fmaxf(bm, v[15]);
+      // running softmax normaliser of this lane's elements
+      if (bm > w.m_t) {
+        w.s_t *= fast_exp2((w.m_t - bm) * LOG2E_F);
+        w.m_t = bm;
       }
-      pool_from_warp(w, queue, s_pool, &s_pool_n, k);
-      wm = m_t;
+      if (w.m_t > -CUDART_INF_F) {
+        // exp(v - m) = 2^(v * log2e - m * log2e); an infinite m (a +inf logit) must give NaN
+        const float c = -w.m_t * LOG2E_F;
+        const u64 c2 = pack_f32x2(c, c), l2 = pack_f32x2(LOG2E_F, LOG2E_F);
+        u64 acc0 = 0ull, acc1 = 0ull;              // two pairs of +0.0f
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+          float x0, x1, x2, x3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(v[i], v[i + 1]), l2, c2), x0, x1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(v[i + 2], v[i + 3]), l2, c2), x2, x3);
+          acc0 = add_f32x2(acc0, pack_f32x2(fast_exp2(x0), fast_exp2(x1)));
+          acc1 = add_f32x2(acc1, pack_f32x2(fast_exp2(x2), fast_exp2(x3)));
+        }
+        float s0, s1;
+        unpack_f32x2(add_f32x2(acc0, acc1), s0, s1);
+        w.s_t += s0 + s1;
+      }
+      refreshed = (t & (t + 1)) == 0;            // after tiles 1, 2, 4, 8, ... of the slice
+      if (refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp);
+      if (__ballot_sync(FULL, bm >= w.thr_f) != 0u)
+        collect_tile(ring + sl * XS_WTILE, v, base, ke, buf, w, lane);
+      // Every lane's loads from the slot have delivered their data (the vote needs every lane's
+      // maximum, and what the collection read has gone into the buffer): the slot can take the
+      // tile XS_RING ahead.
+      __syncwarp();
+      if (lane == 0 && t + XS_RING < nt) issue(t + XS_RING, wt - 1 + XS_RING);
+    }
+    if (nt > 0 && !refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp);
+
+    // ---- the warp's survivors -> the CTA pool; its normaliser -> shared memory ----
+    {
+      // a warp that could not build a threshold (a short slice) brings its ke best keys only
+      if (w.cnt > 2 * ke + 8) cut_back(buf, ke, w, lane);
+      const int n = w.cnt;
+      for (int i = lane; i < n; i += 32) {
+        const u64 key = buf[i];
+        if (key_logit(key) >= w.thr_f) {
+          const int pos = atomicAdd(&s_pool_n, 1);
+          if (pos < XS_POOL) s_pool[pos] = key;
+        }
+      }
+      float wm = w.m_t;
 #pragma unroll
       for (int o = 16; o; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(FULL, wm, o));
-      // thread partial rescaled to the warp maximum; a NaN partial (NaN or +inf logit) propagates
-      ws = (m_t > -CUDART_INF_F || s_t != s_t) ? s_t * exp2f((m_t - wm) * LOG2E_F) : 0.f;
+      // lane partial rescaled to the warp maximum; a NaN partial (NaN or +inf logit) propagates
+      float wsum = (w.m_t > -CUDART_INF_F || w.s_t != w.s_t) ? w.s_t * exp2f((w.m_t - wm) * LOG2E_F) : 0.f;
 #pragma unroll
-      for (int o = 16; o; o >>= 1) ws += __shfl_xor_sync(FULL, ws, o);
-      if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
+      for (int o = 16; o; o >>= 1) wsum += __shfl_xor_sync(FULL, wsum, o);
+      if (lane == 0) { s_m[warp] = wm; s_s[warp] = wsum; }
+    }
+    __syncthreads();
+    if (s_abort) return;
+    if (s_pool_n > XS_POOL) {
+      // the pool cannot hold every survivor (equal logits): each warp brings its ke best only
+      __syncthreads();
+      if (tid == 0) s_pool_n = 0;
+      __syncthreads();
+      cut_back(buf, ke, w, lane);
+      const int n = w.cnt;
+      int pos = 0;
+      if (lane == 0) pos = atomicAdd(&s_pool_n, n);
+      pos = __shfl_sync(FULL, pos, 0);
+      if (lane < n) s_pool[pos + lane] = buf[lane];
       __syncthreads();
     }
 
-    // ---- the chunk's k best keys: four lanes count each candidate's betters (keys are unique) ----
+    // ---- the chunk's ke best keys: four lanes count each candidate's betters (keys are unique) ----
     const int nc = s_pool_n;
     for (int c0 = 0; c0 < nc; c0 += EXP_THREADS / 4) {
       const int ci = c0 + (tid >> 2), q = tid & 3;
       const u64 key = ci < nc ? s_pool[ci] : 0ull;
       int r = 0;
+#pragma unroll 4
       for (int o = q; o < nc; o += 4) r += (s_pool[o] > key) ? 1 : 0;
       r += __shfl_xor_sync(FULL, r, 1);
       r += __shfl_xor_sync(FULL, r, 2);
-      if (q == 0 && ci < nc && r < k) a.part_keys[(size_t)item * a.key_stride + r] = key;
+      if (q == 0 && ci < nc && r < ke) a.part_keys[(size_t)item * a.key_stride + r] = key;
     }
-    if (tid >= nc && tid < k) a.part_keys[(size_t)item * a.key_stride + tid] = 0ull;
+    if (tid < k && tid >= min(nc, ke)) a.part_keys[(size_t)item * a.key_stride + tid] = 0ull;
     if (warp == EXP_WARPS - 1) {
       const float mw = lane < EXP_WARPS ? s_m[lane] : -CUDART_INF_F;
       const float sw = lane < EXP_WARPS ? s_s[lane] : 0.f;
@@ -994,52 +917,134 @@ expand_fused_kernel(FusedArgs a) {
       if (lane == 0) a.part_ms[item] = make_float2(bmx, tot);
     }
 
-    // ---- the last chunk of a sequence runs that sequence's selection.  The barrier orders
-    // this CTA's writes before thread 0's device-scope release; the last arrival acquires. ----
+    // ---- hand-off.  The barrier orders this CTA's writes before thread 0's device-scope
+    // release; the last arrival acquires.  Narrow frontiers count chunks per sequence, wide ones
+    // chunks per row and then rows per sequence. ----
+    const bool two_level = rl.F > XS_TWO_LEVEL;
     __syncthreads();
+    if (lane == 0) { s_wtop[warp] = -CUDART_INF_F; s_wmax[warp] = -CUDART_INF_F; }
     if (tid == 0) {
       s_pool_n = 0;
-      s_thr_cta = 0u;
-      s_anchor = 0ull; s_cnt = 0; s_bad = 0;        // the selection phase's accumulators
-      cuda::atomic_ref<unsigned int, cuda::thread_scope_device> cnt(a.seq_count[rl.b]);
-      const unsigned prev = cnt.fetch_add(1u, cuda::memory_order_acq_rel);
-      s_last = (prev == (unsigned)(rl.F * g.splits) - 1u);
-      if (s_last) cnt.store(0u, cuda::memory_order_relaxed);      // ready for the next layer
+      if (two_level && (unsigned)len == g.pitch) {
+        s_last = 1;                                               // the row's only chunk
+      } else {
+        // the counters add up elements of the line: a row is done at pitch, a narrow frontier at F * pitch
+        cuda::atomic_ref<unsigned int, cuda::thread_scope_device> c(two_level ? a.row_count[row] : a.seq_count[rl.b]);
+        const unsigned target = two_level ? g.pitch : (unsigned)rl.F * g.pitch;
+        const unsigned prev = c.fetch_add((unsigned)len, cuda::memory_order_acq_rel);
+        s_last = (prev + (unsigned)len == target);
+        if (s_last) c.store(0u, cuda::memory_order_relaxed);      // ready for the next layer
+      }
     }
     __syncthreads();
     if (!s_last) continue;
+
     TailSmem sm;
     const int rows_max = a.N - 1;
-    unsigned char *p = smem_raw;
-    sm.stage = reinterpret_cast<u64 *>(p);            p += sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV);
-    sm.row_keys = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * k;
-    sm.score = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max * k;
-    sm.row_t = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max;
-    sm.row_ps = reinterpret_cast<double *>(p);        p += sizeof(double) * rows_max;
-    sm.row_mask = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * a.W;
-    sm.row_m = reinterpret_cast<float *>(p);          p += sizeof(float) * rows_max;
-    sm.row_cnt = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
-    sm.row_off = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
-    sm.state = p;
-    select_tail(a, sm, rl.b, rl.node - rl.j, rl.row0, rl.F, g.splits, &s_anchor, &s_cnt, &s_bad);
+    {
+      unsigned char *p = smem_raw;
+      sm.stage = reinterpret_cast<u64 *>(p);            p += sizeof(u64) * EXP_WARPS * stage_words(k);
+      sm.row_keys = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * k;
+      sm.score = reinterpret_cast<double *>(p);         p += sizeof(double) * rows_max * k;
+      sm.row_mask = reinterpret_cast<u64 *>(p);         p += sizeof(u64) * rows_max * a.W;
+      sm.row_cnt = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
+      sm.row_off = reinterpret_cast<int *>(p);          p += sizeof(int) * rows_max;
+      sm.state = p;
+    }
+    const size_t nb = (size_t)rl.b * a.N;
+    if (two_level) {
+      // ---- this CTA finished a row of a wide frontier: one warp merges it, publishes the result
+      // and counts the row; the CTA that counts the sequence's last row goes on ----
+      if (warp == 0) {
+        u64 key, pmask; double sc;
+        int item0, S;
+        row_chunks(g, row, item0, S);
+        const bool finite = merge_row(a, (size_t)item0, S, k, ke, nb + rl.node, sm.stage, key, sc, pmask);
+        if (!finite) {
+          sc = lane == 0 ? CUDART_NAN : -CUDART_INF;
+          if (lane == 0) atomicOr(a.status, STATUS_NONFINITE);
+        }
+        if (lane < k) {
+          a.row_keys[(size_t)row * a.key_stride + lane] = key;
+          a.row_score[(size_t)row * a.key_stride + lane] = sc;
+        }
+        __syncwarp();
+        if (lane == 0) {
+          cuda::atomic_ref<unsigned int, cuda::thread_scope_device> c(a.seq_count[rl.b]);
+          const unsigned prev = c.fetch_add(1u, cuda::memory_order_acq_rel);
+          s_last_seq = (prev == (unsigned)rl.F - 1u);
+          if (s_last_seq) c.store(0u, cuda::memory_order_relaxed);
+        }
+      }
+      __syncthreads();
+      if (!s_last_seq) continue;
+      // ---- collect the sequence's row results and the parents' mask rows: four loads per thread
+      // go to registers before the first store, so that they share one trip to L2 ----
+      const int C = rl.F * k;
+      for (int c0 = 0; c0 < C; c0 += 4 * EXP_THREADS) {
+        u64 key[4]; double sc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = c0 + u * EXP_THREADS + tid;
+          const int j = c / k, i = c - j * k;
+          key[u] = c < C ? __ldcg(a.row_keys + (size_t)(rl.row0 + j) * a.key_stride + i) : 0ull;
+          sc[u] = c < C ? __ldcg(a.row_score + (size_t)(rl.row0 + j) * a.key_stride + i) : -CUDART_INF;
+        }
+        const int mi = c0 / 4 + tid;                 // the mask words ride along, EXP_THREADS per round
+        const u64 mword = mi < rl.F * a.W ? a.t.mask[(nb + lo) * a.W + mi] : 0ull;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c = c0 + u * EXP_THREADS + tid;
+          if (c >= C) continue;
+          sm.row_keys[c] = key[u];
+          if (sc[u] != sc[u]) { s_bad = 1; sm.score[c] = -CUDART_INF; }
+          else {
+            sm.score[c] = sc[u];
+            // rows are sorted: heads carry the maxima
+            if (c % k == 0 && sc[u] > -CUDART_INF) atomicMax(&s_anchor, f64_ord(sc[u]));
+          }
+        }
+        if (mi < rl.F * a.W) sm.row_mask[mi] = mword;
+      }
+      for (int mi = (C + 4 * EXP_THREADS - 1) / (4 * EXP_THREADS) * EXP_THREADS + tid; mi < rl.F * a.W; mi += EXP_THREADS)
+        sm.row_mask[mi] = a.t.mask[(nb + lo) * a.W + mi];
+    } else {
+      // ---- this CTA finished the sequence: one warp per row ----
+      for (int j = warp; j < rl.F; j += EXP_WARPS) {
+        u64 key, pmask; double sc;
+        int item0, S;
+        row_chunks(g, rl.row0 + j, item0, S);
+        const bool finite = merge_row(a, (size_t)item0, S, k, ke, nb + lo + j, sm.stage + warp * stage_words(k), key, sc,
+                                      pmask);
+        if (!finite && lane == 0) { s_bad = 1; atomicOr(a.status, STATUS_NONFINITE); }
+        if (lane < k) {
+          sm.row_keys[j * k + lane] = key;
+          sm.score[j * k + lane] = sc;
+        }
+        if (lane < a.W) sm.row_mask[j * a.W + lane] = pmask;
+        if (lane == 0 && sc > -CUDART_INF) atomicMax(&s_anchor, f64_ord(sc));
+      }
+    }
+    __syncthreads();
+    if (s_bad) {             // a frontier row was not finite: this sequence adds nothing
+      if (tid == 0) a.t.layer_off[rl.b * a.lo_stride + a.d + 2] = n_before;
+    } else {
+      select_and_append(a, sm, rl.b, lo, rl.F, n_before, &s_anchor, &s_ecnt);
+    }
     __syncthreads();     // the next chunk's bulk copies land in the memory the selection phase just used
+    if (tid == 0) { s_anchor = 0ull; s_ecnt = 0; s_bad = 0; }
   }
 }
 
 size_t fused_smem_bytes(const talon_ctx *c) {
   const size_t rows = c->p.budget - 1, k = c->k_cap, W = c->W;
-  const size_t tail = sizeof(u64) * EXP_WARPS * (32 * k + FX_SURV) + rows * k * (8 + 8 + 1) +
-                      rows * (8 + 8 + 8 * W + 4 + 4 + 4) + 16;
-  const size_t ring = sizeof(float) * FX_RING * EXP_TILE;       // the two phases share the space
+  const size_t tail = sizeof(u64) * EXP_WARPS * (FX_MAX_SPLITS * k + FX_SURV + k) + rows * k * (8 + 8 + 1) +
+                      rows * (8 * W + 4 + 4) + 16;
+  const size_t ring = sizeof(float) * EXP_WARPS * XS_RING * XS_WTILE;       // the two phases share the space
   return tail > ring ? tail : ring;
 }
 
 }  // namespace
-
-int fused_max_splits(int key_stride) {
-  (void)key_stride;
-  return FX_MAX_SPLITS;
-}
 
 talon_status expand_fused_setup(talon_ctx *c) {
   const size_t bytes = fused_smem_bytes(c);
@@ -1062,15 +1067,14 @@ talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float 
   a.t = *t; a.lo_stride = c->p.max_depth + 2;
   a.B = c->B; a.N = c->p.budget; a.W = c->W; a.V = c->p.vocab; a.d = c->layers_run; a.k = c->k_cap;
   a.key_stride = c->key_stride;
-  a.max_splits = fused_max_splits(c->key_stride);
-  long long max_items = (long long)rows_bound * a.max_splits;
+  a.max_split = c->expand_max_split;
+  long long max_items = (long long)rows_bound * FX_MAX_SPLITS;
   int grid = c->fused_grid;
   if (max_items < grid) grid = (int)max_items;
   if (grid < 1) grid = 1;
-  a.target_items = grid;
-  a.items_cap = c->items_cap;
   a.root_topk = c->p.root_topk; a.init_layers = c->p.init_layers; a.log_mu = c->log_mu;
-  a.part_keys = c->d_part_keys; a.part_ms = c->d_part_ms; a.seq_count = c->d_seq_count; a.status = c->d_status;
+  a.part_keys = c->d_part_keys; a.part_ms = c->d_part_ms; a.row_keys = c->d_row_keys; a.row_score = c->d_row_score;
+  a.row_count = c->d_row_count; a.seq_count = c->d_seq_count; a.status = c->d_status;
   {
     LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
     launch_kernel(c, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c), st, a);

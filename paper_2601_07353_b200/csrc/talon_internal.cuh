@@ -26,11 +26,9 @@ constexpr int MAX_BUDGET = 128;
 constexpr int MAX_BATCH = 1024;
 constexpr int SEL_THREADS = 512;
 // fused expansion kernel (k <= 32)
-constexpr int FX_QCAP = 128;               // keys a warp's queue can hold
+constexpr int FX_QCAP = 128;               // keys a warp's candidate buffer can hold
 constexpr int FX_SURV = 64;                // keys of a row that may pass the merge bound before the slow path
-constexpr int FX_MAX_SPLITS = 32;          // chunks per row, at most (one lane per chunk in the merge)
-constexpr int FX_RING = 3;                 // 16 KB tiles in flight per CTA on the streaming path
-constexpr int FX_POOL = 256;               // candidates a CTA can pool for one chunk
+constexpr int FX_MAX_SPLITS = 16;          // chunks per row, at most (one lane per chunk in the merge)
 
 // Order-preserving map fp32 -> u32 (larger float <=> larger integer; -inf > 0).
 __host__ __device__ inline uint32_t f32_ord(float f) {
@@ -119,9 +117,11 @@ struct talon_ctx {
   float2 *d_part_ms;                 // [items_cap]              per-chunk (max, sum exp)
   unsigned long long *d_row_keys;    // [rows_cap, key_stride]   per-row top-k
   double *d_row_lse;                 // [rows_cap]               per-row log-sum-exp
+  double *d_row_score;               // [rows_cap, key_stride]   per-row candidate scores (fused kernel, wide frontiers)
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int expand_max_split;              // fused kernel: chunks a row is cut into at most when the grid has room
   int attn_min_tiles;                // split-KV: key tiles a CTA should at least own
   int pdl;                           // programmatic stream serialization: 1 on, 0 off, -1 on for small batches
   // verification workspace
