@@ -62,22 +62,26 @@ def attention_flops(prefix_len: int, n_nodes: int, n_q_heads: int, head_dim: int
     return 4 * head_dim * n_q_heads * n_nodes * (prefix_len + n_nodes)
 
 
-def captured_traffic_ratio(kernel: str):
-    """DRAM bytes per algorithmic byte of ``kernel`` from its last ncu capture, or None.
+def source_hash(root: str, sources: Sequence[str]) -> str:
+    h = hashlib.sha256()
+    for rel in sources:
+        with open(os.path.join(root, rel), "rb") as src:
+            h.update(src.read())
+    return h.hexdigest()
 
-    ``traffic_capture.json`` records, per kernel, the ratio measured under ncu together with a
-    hash of the kernel's source files at that time; a kernel whose source changed since then has
-    no valid counters, so None is returned and the benchmark reports ``traffic`` as null."""
-    here = os.path.dirname(os.path.abspath(__file__))
+
+def captured_traffic_ratio(root: str, kernel: str, workload: str):
+    """DRAM bytes per algorithmic byte of ``kernel`` on ``workload`` from its last ncu capture, or None.
+
+    ``profiles/traffic_capture.json`` under ``root`` records, per kernel, the ratios measured under
+    ncu (one per workload) together with a hash of the kernel's source files at that time; a kernel
+    whose source changed since then has no valid counters, so None is returned and the benchmark
+    reports ``traffic`` as null."""
     try:
-        with open(os.path.join(here, "traffic_capture.json")) as f:
+        with open(os.path.join(root, "profiles", "traffic_capture.json")) as f:
             rec = json.load(f)[kernel]
-        h = hashlib.sha256()
-        for rel in rec["sources"]:
-            with open(os.path.join(os.path.dirname(here), rel), "rb") as src:
-                h.update(src.read())
-        if h.hexdigest() != rec["sha256"]:
+        if source_hash(root, rec["sources"]) != rec["sha256"]:
             return None
-        return float(rec["dram_bytes_per_algorithmic_byte"])
-    except (OSError, KeyError, ValueError):
+        return float(rec["dram_bytes_per_algorithmic_byte"][workload])
+    except (OSError, KeyError, ValueError, TypeError):
         return None

@@ -31,21 +31,25 @@ def test_peaks_fall_back_when_the_file_is_missing(tmp_path):
     assert p["source"] == "measured" and p["hbm_gbs"] == 6000.0 and p["bf16_tflops_sustained"] == 1500.0
 
 
-def test_traffic_ratio_is_void_once_the_kernel_source_changed(tmp_path, monkeypatch):
-    import json, os, shutil
-    pkg = os.path.dirname(roofline.__file__)
-    rec = json.load(open(os.path.join(pkg, "traffic_capture.json")))
-    assert "expand_rows" in rec and len(rec["expand_rows"]["sha256"]) == 64
-    # a record whose hash does not match the sources gives no traffic figure
-    fake_pkg = tmp_path / "paper_2601_07353_b200"
-    (fake_pkg / "csrc").mkdir(parents=True)
-    for rel in rec["expand_rows"]["sources"]:
-        shutil.copy(os.path.join(os.path.dirname(pkg), rel), tmp_path / rel)
-    shutil.copy(os.path.join(pkg, "traffic_capture.json"), fake_pkg / "traffic_capture.json")
-    monkeypatch.setattr(roofline, "__file__", str(fake_pkg / "roofline.py"))
-    same = roofline.captured_traffic_ratio("expand_rows")
-    with open(tmp_path / rec["expand_rows"]["sources"][0], "a") as f:
+def test_traffic_ratio_is_void_once_the_kernel_source_changed(tmp_path):
+    import json
+    (tmp_path / "profiles").mkdir()
+    (tmp_path / "csrc").mkdir()
+    (tmp_path / "csrc" / "k.cu").write_text("__global__ void k() {}\n")
+    rec = {"expand_rows": {"sources": ["csrc/k.cu"], "sha256": roofline.source_hash(str(tmp_path), ["csrc/k.cu"]),
+                           "dram_bytes_per_algorithmic_byte": {"llama8b": 1.05}}}
+    (tmp_path / "profiles" / "traffic_capture.json").write_text(json.dumps(rec))
+    assert roofline.captured_traffic_ratio(str(tmp_path), "expand_rows", "llama8b") == 1.05
+    assert roofline.captured_traffic_ratio(str(tmp_path), "expand_rows", "longctx") is None      # no capture on that workload
+    assert roofline.captured_traffic_ratio(str(tmp_path), "no_such_kernel", "llama8b") is None
+    with open(tmp_path / "csrc" / "k.cu", "a") as f:
         f.write("// changed\n")
-    assert roofline.captured_traffic_ratio("expand_rows") is None
-    assert roofline.captured_traffic_ratio("no_such_kernel") is None
-    assert same is None or same > 0.9
+    assert roofline.captured_traffic_ratio(str(tmp_path), "expand_rows", "llama8b") is None
+
+
+def test_the_committed_traffic_record_names_existing_sources():
+    import json, os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(roofline.__file__)))
+    rec = json.load(open(os.path.join(root, "profiles", "traffic_capture.json")))
+    for kernel, r in rec.items():
+        assert len(r["sha256"]) == 64 and all(os.path.exists(os.path.join(root, s)) for s in r["sources"]), kernel
