@@ -267,7 +267,8 @@ talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const
  * fixed memory pool, or in a part of a serving loop where allocating is not allowed (it
  * synchronises the device and may fail when memory is tight), can use this call instead for the
  * first half of the greedy verification: t_i = argmax of target-logit row i, lowest id among
- * equal maxima, -1 for a row that holds only NaN.  It needs no context and calls no cudaMalloc,
+ * equal maxima.  A NaN never competes, wherever it sits in the row; a row that holds nothing but
+ * NaN gives -1 (a row of -inf only gives token 0, like any other row of equal values).  It needs no context and calls no cudaMalloc,
  * cudaFree or any other allocating routine; its scratch (one 8-byte key per row) is a fixed
  * array inside the library image, TALON_NOALLOC_MAX_ROWS * 8 bytes on every GPU that loads the
  * library, held until the process exits.
@@ -276,8 +277,8 @@ talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const
  *  n_rows        0 .. TALON_NOALLOC_MAX_ROWS; more returns TALON_ERR_CAPACITY, nothing enqueued
  *  target_tok    device [n_rows]
  * Runs on the current device; enqueues three kernels on `stream` and returns.  The first call on
- * a device looks up the array's device address (cudaGetSymbolAddress) and the SM count; make
- * that first call outside any stream capture.  Every call clears the rows it uses first, since
+ * a device looks up the array's device address (cudaGetSymbolAddress) and the SM count, under a
+ * lock, so host threads may race to it; make that first call outside any stream capture.  Every call clears the rows it uses first, since
  * the array keeps the previous call's keys.  All calls share the one array: two calls that can
  * overlap on the GPU (different streams without an ordering between them) race. */
 #define TALON_NOALLOC_MAX_ROWS 8192

@@ -8,6 +8,7 @@
 #include <math_constants.h>
 
 #include <cstdio>
+#include <mutex>
 
 #include "talon_internal.cuh"
 
@@ -51,8 +52,11 @@ noalloc_argmax_kernel(const float *logits, int64_t row_stride, int V, int n_rows
         for (int e = 0; e < 4; ++e) x[e] = (idx + e < end) ? __ldcs(rowp + idx + e) : -CUDART_INF_F;
       }
 #pragma unroll
-      for (int e = 0; e < 4; ++e)   // strict > keeps the lowest index among equal values
-        if (idx + e < end && (x[e] > bestv || besti == 0xFFFFFFFFu)) { bestv = x[e]; besti = (uint32_t)(idx + e); }
+      for (int e = 0; e < 4; ++e)   // strict > keeps the lowest index among equal values; a NaN never competes
+        if (idx + e < end && x[e] == x[e] && (x[e] > bestv || besti == 0xFFFFFFFFu)) {
+          bestv = x[e];
+          besti = (uint32_t)(idx + e);
+        }
     }
     unsigned long long key = (besti == 0xFFFFFFFFu) ? 0ull : cand_key(bestv, besti);
 #pragma unroll
@@ -86,6 +90,7 @@ struct DeviceSlot {
   int sm_count;
 };
 DeviceSlot g_slots[NA_MAX_DEVICES];
+std::mutex g_slots_lock;       // two host threads may make the first call on a device at once
 
 }  // namespace
 }  // namespace talon
@@ -106,7 +111,9 @@ extern "C" talon_status talon_target_argmax_noalloc(const float *target_logits, 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES) return TALON_ERR_CUDA;
   DeviceSlot &slot = g_slots[dev];
-  if (!slot.ready) {
+  {
+    std::lock_guard<std::mutex> hold(g_slots_lock);
+    if (!slot.ready) {
     // In host code the array's name is only a handle: the device address has to be asked for,
     // with the device that will run the kernels current.
     void *p = nullptr;
@@ -120,6 +127,7 @@ extern "C" talon_status talon_target_argmax_noalloc(const float *target_logits, 
     slot.scratch = static_cast<unsigned long long *>(p);
     slot.sm_count = sms;
     slot.ready = true;
+    }
   }
   cudaStream_t st = (cudaStream_t)stream;
   // chunks per row: enough items to fill the GPU, chunks a multiple of 1024 elements

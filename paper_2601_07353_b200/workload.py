@@ -66,19 +66,35 @@ def _bf16(x32: torch.Tensor) -> torch.Tensor:
     return x32.to(torch.bfloat16)
 
 
+def logit_rows(B: int, N: int, V: int, row_pad: int, dev) -> torch.Tensor:
+    """[B, N, V] fp32 rows that start 16 bytes aligned: the row stride is V rounded up to a multiple
+    of four elements plus ``row_pad``; what lies between the rows holds NaN, which no kernel may use."""
+    assert row_pad % 4 == 0
+    stride = (V + 3) // 4 * 4 + row_pad
+    if stride == V:
+        return torch.zeros(B, N, V, dtype=torch.float32, device=dev)
+    buf = torch.full((B, N, stride), float("nan"), dtype=torch.float32, device=dev)
+    rows = buf[:, :, :V]
+    rows.zero_()
+    return rows
+
+
 def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAULT_SEED,
-                   seq_ids: Optional[Sequence[int]] = None, with_verify: bool = True) -> Workload:
+                   seq_ids: Optional[Sequence[int]] = None, with_verify: bool = True, row_pad: int = 0,
+                   prefix_lens: Optional[Sequence[int]] = None) -> Workload:
+    """``row_pad`` widens the logit rows' stride (NaN padding); ``prefix_lens`` overrides the hashed
+    prefix lengths of the sequences (the generated K/V of a sequence are cut to that length)."""
     dev = talon.device
     seq_ids = list(range(cfg.batch)) if seq_ids is None else list(seq_ids)
     B, N, V = len(seq_ids), cfg.budget, cfg.vocab
-    assert V % 4 == 0, "dense logit rows must stay 16-byte aligned"
     i32 = dict(dtype=torch.int32, device=dev)
     root = torch.tensor([synth.root_token(cfg, seed, s) for s in seq_ids], **i32)
-    plens = [synth.prefix_len(cfg, seed, s) for s in seq_ids]
+    plens = [synth.prefix_len(cfg, seed, s) for s in seq_ids] if prefix_lens is None else [int(x) for x in prefix_lens]
+    assert len(plens) == B
     prefix_len = torch.tensor(plens, **i32)
     starts = np.concatenate([[0], np.cumsum(plens)[:-1]]).astype(np.int64)
     kv_start = torch.tensor(starts, dtype=torch.int64, device=dev)
-    draft = torch.zeros(B, N, V, dtype=torch.float32, device=dev)
+    draft = logit_rows(B, N, V, row_pad, dev)
     tree = talon.alloc_tree(B)
 
     talon.reset(tree, root, prefix_len)
@@ -109,7 +125,7 @@ def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAU
     bf = dict(dtype=torch.bfloat16, device=dev)
     total = int(sum(plens))
     wl = Workload(cfg, seed, seq_ids, root, prefix_len, kv_start, max(plens), draft,
-                  target=torch.zeros((B, N, V) if with_verify else (1, 1, 4), dtype=torch.float32, device=dev),
+                  target=logit_rows(B, N, V, row_pad, dev) if with_verify else torch.zeros(1, 1, 4, dtype=torch.float32, device=dev),
                   q=torch.zeros(B, N, Hq, Dh, **bf), k_prefix=torch.zeros(max(total, 1), Hkv, Dh, **bf),
                   v_prefix=torch.zeros(max(total, 1), Hkv, Dh, **bf), k_tree=torch.zeros(B, N, Hkv, Dh, **bf),
                   v_tree=torch.zeros(B, N, Hkv, Dh, **bf), tree=tree, out=torch.zeros(B, N, Hq, Dh, **bf),
