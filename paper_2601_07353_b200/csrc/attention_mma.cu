@@ -332,7 +332,7 @@ static int attn_m_blocks(const talon_ctx *c) {
 
 size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems) {
   const int mb = attn_m_blocks(c);
-  long long ctas = (long long)c->p.batch_max * c->p.n_kv_heads * mb;
+  long long ctas = 2LL * c->p.batch_max * c->p.n_kv_heads * mb;       // room for two key ranges per CTA slot
   if (ctas < 2LL * c->sm_count) ctas = 2LL * c->sm_count;
   *ml_elems = (size_t)ctas * AT_BM;
   return (size_t)ctas * AT_BM * AT_D;
@@ -369,6 +369,18 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
       const int by_tiles = (tiles + c->attn_min_tiles - 1) / c->attn_min_tiles;
       if (sp > by_tiles) sp = by_tiles;
       if (sp < 1) sp = 1;
+    } else if (ctas % c->sm_count) {
+      // More CTAs than SMs and a ragged last wave: halving the key ranges can fill it (512 CTAs on
+      // 148 SMs are 4 waves of 257 tiles, 1024 half CTAs are 7 waves of 129).  Cost model in key
+      // tiles: waves x (tiles per CTA + 2 for the prologue and epilogue), plus what merging the
+      // partial results costs, about one tile per 24 CTAs per SM.
+      const long long sm = c->sm_count;
+      auto cost = [&](int s) {
+        const long long n = (long long)ctas * s;
+        const long long waves = (n + sm - 1) / sm;
+        return waves * ((tiles + s - 1) / s + 2) + (s > 1 ? n / (24 * sm) + 3 : 0);
+      };
+      if (tiles >= 32 && cost(2) < cost(1)) sp = 2;
     }
     while (sp > 1 && (size_t)a.m_blocks * c->B * a.Hkv * sp * AT_BM > c->attn_ml_elems) --sp;
     a.splits = sp;

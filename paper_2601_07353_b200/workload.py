@@ -81,10 +81,14 @@ def logit_rows(B: int, N: int, V: int, row_pad: int, dev) -> torch.Tensor:
 
 def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAULT_SEED,
                    seq_ids: Optional[Sequence[int]] = None, with_verify: bool = True, row_pad: int = 0,
-                   prefix_lens: Optional[Sequence[int]] = None) -> Workload:
+                   prefix_lens: Optional[Sequence[int]] = None, host_inputs: bool = False) -> Workload:
     """``row_pad`` widens the logit rows' stride (NaN padding); ``prefix_lens`` overrides the hashed
-    prefix lengths of the sequences (the generated K/V of a sequence are cut to that length)."""
+    prefix lengths of the sequences (the generated K/V of a sequence are cut to that length);
+    ``host_inputs`` generates every input with NumPy on the host and uploads it (bit-identical to
+    the device generator), so that the only kernels the GPU runs are the library's."""
     dev = talon.device
+    gen_dev = None if host_inputs else dev
+    up = (lambda x: torch.from_numpy(np.ascontiguousarray(x))) if host_inputs else (lambda x: x)
     seq_ids = list(range(cfg.batch)) if seq_ids is None else list(seq_ids)
     B, N, V = len(seq_ids), cfg.budget, cfg.vocab
     i32 = dict(dtype=torch.int32, device=dev)
@@ -113,7 +117,7 @@ def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAU
             any_active = True
             paths = node_paths(token[bi], parent[bi], n)
             for i in range(max(done_rows[bi], int(lo[bi, d])), int(lo[bi, d + 1])):
-                draft[bi, i] = synth.draft_logits_row(cfg, seed, s, paths[i], device=dev)
+                draft[bi, i] = up(synth.draft_logits_row(cfg, seed, s, paths[i], device=gen_dev))
             done_rows[bi] = int(lo[bi, d + 1])
         if not any_active:
             break
@@ -141,10 +145,10 @@ def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAU
         n = int(n_nodes[bi])
         paths = node_paths(token[bi], parent[bi], n)
         for i in range(n):
-            wl.target[bi, i] = synth.target_logits_row(cfg, seed, s, paths[i], device=dev)
-        wl.q[bi] = _bf16(synth.qkv_block(seed, synth.STREAM_Q, s, N * Hq * Dh, dev)).view(N, Hq, Dh)
-        wl.k_tree[bi] = _bf16(synth.qkv_block(seed, synth.STREAM_KT, s, N * Hkv * Dh, dev)).view(N, Hkv, Dh)
-        wl.v_tree[bi] = _bf16(synth.qkv_block(seed, synth.STREAM_VT, s, N * Hkv * Dh, dev)).view(N, Hkv, Dh)
+            wl.target[bi, i] = up(synth.target_logits_row(cfg, seed, s, paths[i], device=gen_dev))
+        wl.q[bi] = _bf16(up(synth.qkv_block(seed, synth.STREAM_Q, s, N * Hq * Dh, gen_dev))).view(N, Hq, Dh)
+        wl.k_tree[bi] = _bf16(up(synth.qkv_block(seed, synth.STREAM_KT, s, N * Hkv * Dh, gen_dev))).view(N, Hkv, Dh)
+        wl.v_tree[bi] = _bf16(up(synth.qkv_block(seed, synth.STREAM_VT, s, N * Hkv * Dh, gen_dev))).view(N, Hkv, Dh)
         L = plens[bi]
         if L:
             a = int(starts[bi])
@@ -152,8 +156,8 @@ def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAU
             for t0 in range(0, L, step):
                 t1 = min(L, t0 + step)
                 cnt, off = (t1 - t0) * Hkv * Dh, t0 * Hkv * Dh
-                wl.k_prefix[a + t0:a + t1] = _bf16(synth.qkv_block(seed, synth.STREAM_K, s, cnt, dev, off)).view(-1, Hkv, Dh)
-                wl.v_prefix[a + t0:a + t1] = _bf16(synth.qkv_block(seed, synth.STREAM_V, s, cnt, dev, off)).view(-1, Hkv, Dh)
+                wl.k_prefix[a + t0:a + t1] = _bf16(up(synth.qkv_block(seed, synth.STREAM_K, s, cnt, gen_dev, off))).view(-1, Hkv, Dh)
+                wl.v_prefix[a + t0:a + t1] = _bf16(up(synth.qkv_block(seed, synth.STREAM_V, s, cnt, gen_dev, off))).view(-1, Hkv, Dh)
     return wl
 
 
