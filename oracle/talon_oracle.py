@@ -33,6 +33,10 @@ What follows which passage:
   efficiency delta = N_q / N_p, the mean accepted tokens tau = L / N_p and the speed-up
   R = tau / (1 + c delta) of Section 5.3 and its derivation in the appendix.
 
+* ``expand_static`` / ``prune_static`` -- Algorithm 1 (the static tree the paper compares with): at
+  every depth 0..D each parent proposes its Top-K tokens, the K x K pool is cut to the K best path
+  probabilities, which join the tree and become the next parents; at the end the tree is pruned to
+  the N best path probabilities.
 Readings taken where the paper is silent (all listed in the design notes): the budget N
 counts the root; ``max_depth`` is an extra stop; a per-parent candidate cap ``cand_topk``
 (== vocabulary size gives the paper's full pool); ties go to the lower parent index, then
@@ -195,6 +199,61 @@ def expand(root_token: int, logits_fn: Callable[[List[int]], np.ndarray], p: Par
         rows = [logits_fn(path_tokens(tree, v)) for v in tree.frontier]
         expand_layer(tree, rows, p)
     return tree
+
+
+def expand_static(root_token: int, logits_fn: Callable[[List[int]], np.ndarray], width: int, depth: int) -> Tree:
+    """Algorithm 1 up to its pruning step: for d = 0..depth every parent v of the layer proposes
+    C_v = Top-K of its next-token distribution with p(u) = p(v) * P(u | v); the pool S_d of all
+    proposals is cut to its K best by p(u); those join the tree and are the parents of the next
+    layer.  The tree holds 1 + K * (depth + 1) nodes (fewer if a vocabulary is smaller than K).
+    Ties and storage order as everywhere in this file."""
+    cap = 1 + width * (depth + 1)
+    tree = new_tree(root_token, cap, depth + 1)
+    parents = [0]
+    for d in range(depth + 1):
+        pool = []
+        for v in parents:
+            z32 = logits_fn(path_tokens(tree, v))
+            lse = log_softmax_norm(z32)
+            for w in row_topk(z32, width):                                  # C_v
+                logp = float(np.float64(z32[w])) - lse
+                if logp > -np.inf:
+                    pool.append((float(tree.score[v]) + logp, int(v), int(w)))   # p(u) = p(v) P(u | v)
+        nxt = sorted(pool, key=lambda u: (-u[0], u[1], u[2]))[:width]      # Top-K of S_d by p(u)
+        nxt.sort(key=lambda u: (u[1], u[2]))
+        parents = []
+        for s, v, w in nxt:
+            i = tree.n_nodes
+            tree.token[i], tree.parent[i], tree.depth[i], tree.score[i] = w, v, tree.depth[v] + 1, s
+            tree.mask[i] = tree.mask[v]
+            tree.mask[i, i // 64] |= np.uint64(1) << np.uint64(i % 64)
+            tree.n_nodes += 1
+            parents.append(i)
+        tree.layer_off.append(tree.n_nodes)
+        tree.layers_run += 1
+    return tree
+
+
+def prune_static(tree: Tree, keep: int) -> Tree:
+    """Algorithm 1's last step: T <- Top-N(T by p(u)).  Equal scores go to the lower node index, so
+    a kept node's parent (whose probability is at least as large and whose index is lower) is
+    kept too.  The survivors keep their relative order; parents and mask bits are renumbered."""
+    n = tree.n_nodes
+    order = sorted(range(n), key=lambda i: (-float(tree.score[i]), i))[:keep]
+    kept = sorted(order)
+    new_of = {old: new for new, old in enumerate(kept)}
+    out = new_tree(int(tree.token[0]), tree.budget, tree.max_depth)
+    out.n_nodes = len(kept)
+    for new, old in enumerate(kept):
+        out.token[new], out.depth[new], out.score[new] = tree.token[old], tree.depth[old], tree.score[old]
+        out.parent[new] = -1 if tree.parent[old] < 0 else new_of[int(tree.parent[old])]
+        out.mask[new] = 0
+        for j in range(n):
+            if (int(tree.mask[old, j // 64]) >> (j % 64)) & 1:
+                out.mask[new, new_of[j] // 64] |= np.uint64(1) << np.uint64(new_of[j] % 64)
+    out.layers_run = tree.layers_run
+    out.layer_off = [sum(1 for i in kept if tree.depth[i] < d) for d in range(tree.layers_run + 2)]
+    return out
 
 
 def dense_mask(tree: Tree) -> np.ndarray:
