@@ -129,6 +129,19 @@ int32_t talon_layers_run(const talon_ctx *ctx);
 talon_status talon_build_tree(talon_ctx *ctx, const talon_tree *tree, uint8_t *dense_mask,
                               void *stream);
 
+/* The static tree the paper compares with (Algorithm 1, "Static Tree Construction") on the same
+ * kernels.  Its depth loop is talon_expand_layer of a context created with
+ *   budget = 1 + K * (D + 1), root_topk = cand_topk = K, max_depth = init_layers = D + 1:
+ * every layer then takes each parent's Top-K tokens, pools the K x K proposals and keeps the K
+ * best path probabilities as the next parents.  This call is the algorithm's last step,
+ * T <- Top-N(T by p(u)): of every sequence's tree the `keep` nodes with the largest path scores
+ * stay (equal scores: the lower node index, so parents outlive their children), in their old
+ * order; parent links, ancestor-mask bits, layer offsets and n_nodes are renumbered in place.
+ * Call talon_build_tree afterwards (positions, sentinels of the freed slots).
+ *  keep  >= 1; a tree that is not larger is left as it is
+ * Enqueues one kernel; no synchronisation. */
+talon_status talon_prune_tree(talon_ctx *ctx, const talon_tree *tree, int32_t keep, void *stream);
+
 /* Tree attention of the verification forward (Appendix B): query node i of sequence b and
  * query head h attends to all L_b prefix keys and to the tree keys j with mask bit (i, j)
  * set, softmax(sm_scale * q.k) in fp32, times V, accumulated in fp32, written as bf16.

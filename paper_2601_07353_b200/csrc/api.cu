@@ -216,6 +216,12 @@ talon_status talon_build_tree(talon_ctx *c, const talon_tree *t, uint8_t *dense_
   return talon::launch_build(c, t, dense_mask, (cudaStream_t)stream);
 }
 
+talon_status talon_prune_tree(talon_ctx *c, const talon_tree *t, int32_t keep, void *stream) {
+  if (!c || !tree_complete(t)) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || keep < 1) return TALON_ERR_INVALID_ARG;
+  return talon::launch_prune(c, t, keep, (cudaStream_t)stream);
+}
+
 talon_status talon_tree_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *k_prefix,
                                   const void *v_prefix, const void *k_tree, const void *v_tree,
                                   const int64_t *kv_start, int64_t kv_tokens, int64_t kv_stride_t,

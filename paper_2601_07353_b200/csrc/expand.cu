@@ -636,9 +636,80 @@ __global__ void build_tree_kernel(talon_tree t, const int32_t *prefix_len, uint8
   }
 }
 
+// Last step of Algorithm 1 (static tree construction): T <- Top-N(T by p(u)).  One CTA per
+// sequence, one thread per node.  A node's rank is the number of nodes with a larger score, or
+// the same score and a lower index, so a kept node's parent (score at least as large, index
+// lower) is kept too; the survivors keep their order, parents and mask bits are renumbered, the
+// layer offsets recounted.  Slots past the new size are left to talon_build_tree.
+__global__ void __launch_bounds__(MAX_BUDGET)
+prune_tree_kernel(talon_tree t, int B, int N, int W, int lo_stride, int keep) {
+  __shared__ double s_score[MAX_BUDGET];
+  __shared__ int s_new[MAX_BUDGET];          // new index of a kept node, -1 for a dropped one
+  __shared__ int s_depth[MAX_BUDGET];
+  __shared__ unsigned s_keep[MAX_BUDGET / 32];
+  pdl_enter();
+  const int b = blockIdx.x, i = threadIdx.x, lane = i & 31, warp = i >> 5;
+  const int n = t.n_nodes[b];
+  const size_t nb = (size_t)b * N;
+  const bool live = i < n;
+  const double sc = live ? t.score[nb + i] : -CUDART_INF;
+  const int tok = live ? t.token[nb + i] : -1, par = live ? t.parent[nb + i] : -1, dep = live ? t.depth[nb + i] : -1;
+  unsigned long long mk[2] = {0ull, 0ull};
+  if (live)
+    for (int w = 0; w < W; ++w) mk[w] = t.mask[(nb + i) * W + w];
+  s_score[i] = sc;
+  __syncthreads();
+  int rank = 0;
+  for (int j = 0; j < n; ++j) rank += (s_score[j] > sc || (s_score[j] == sc && j < i)) ? 1 : 0;
+  const bool kept = live && rank < keep;
+  const unsigned bal = __ballot_sync(0xFFFFFFFFu, kept);
+  if (lane == 0) s_keep[warp] = bal;
+  __syncthreads();
+  int before = __popc(bal & ((1u << lane) - 1u));
+  for (int w = 0; w < warp; ++w) before += __popc(s_keep[w]);
+  int total = 0;
+  for (int w = 0; w < MAX_BUDGET / 32; ++w) total += __popc(s_keep[w]);
+  s_new[i] = kept ? before : -1;
+  s_depth[i] = kept ? dep : 0x7FFFFFFF;
+  __syncthreads();
+  if (kept) {
+    const int ni = before;
+    t.token[nb + ni] = tok;
+    t.parent[nb + ni] = par < 0 ? -1 : s_new[par];
+    t.depth[nb + ni] = dep;
+    t.score[nb + ni] = sc;
+    unsigned long long nm[2] = {0ull, 0ull};
+    for (int w = 0; w < W; ++w) {
+      unsigned long long bits = mk[w];
+      while (bits) {
+        const int j = w * 64 + __ffsll((long long)bits) - 1;
+        bits &= bits - 1ull;
+        const int nj = s_new[j];
+        if (nj >= 0) nm[nj >> 6] |= 1ull << (nj & 63);
+      }
+    }
+    for (int w = 0; w < W; ++w) t.mask[(nb + ni) * W + w] = nm[w];
+  }
+  // layer_off[d] = kept nodes of depth < d (kept nodes stay sorted by depth)
+  for (int d = i; d < lo_stride; d += MAX_BUDGET) {
+    int c = 0;
+    for (int j = 0; j < n; ++j) c += s_depth[j] < d ? 1 : 0;
+    t.layer_off[b * lo_stride + d] = c;
+  }
+  if (i == 0) t.n_nodes[b] = total;
+}
+
 // ---------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------
+talon_status launch_prune(talon_ctx *c, const talon_tree *t, int keep, cudaStream_t st) {
+  LaunchTimer lt(c, TALON_K_BUILD, st);
+  launch_kernel(c, prune_tree_kernel, dim3(c->B), dim3(MAX_BUDGET), 0, st, *t, c->B, c->p.budget, c->W,
+                c->p.max_depth + 2, keep);
+  c->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? TALON_OK : TALON_ERR_CUDA;
+}
+
 static int frontier_upper_bound(const talon_ctx *c, int d) {
   // host-side bound on rows per sequence at layer d (the device knows the real sizes)
   long long f = 1;

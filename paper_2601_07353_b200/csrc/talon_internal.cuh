@@ -201,6 +201,7 @@ talon_status launch_reset(talon_ctx *c, const talon_tree *t, const int32_t *root
 talon_status launch_expand(talon_ctx *c, const talon_tree *t, const float *logits,
                            int64_t row_stride, int rows_per_seq, int layout, cudaStream_t st);
 talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cudaStream_t st);
+talon_status launch_prune(talon_ctx *c, const talon_tree *t, int keep, cudaStream_t st);
 talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp,
                               const void *vp, const void *kt, const void *vt,
                               const int64_t *kv_start, int64_t kv_tokens, int64_t stride_t, int64_t stride_h,

@@ -45,6 +45,7 @@ _lib.talon_reset.argtypes = [_vp, _TP, _vp, _vp, _i32, _vp]
 _lib.talon_expand_layer.argtypes = [_vp, _TP, _vp, _i64, _i32, _i32, _vp]
 _lib.talon_layers_run.argtypes = [_vp]
 _lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
+_lib.talon_prune_tree.argtypes = [_vp, _TP, _i32, _vp]
 _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_accept_sample.argtypes = [_vp, _TP, _vp, _i64, C.c_double, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -66,7 +67,7 @@ _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
            "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
-           "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit"):
+           "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit", "talon_prune_tree"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
@@ -74,7 +75,7 @@ EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer"
             "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
             "talon_kernel_name",
             "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample",
-            "talon_commit"]
+            "talon_commit", "talon_prune_tree"]
 NOALLOC_MAX_ROWS = 8192
 N_KERNELS = 11
 KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
@@ -198,6 +199,11 @@ class Talon:
         ts = tree.struct()
         _check(_lib.talon_build_tree(self._ctx, C.byref(ts), _ptr(dense_mask), _stream(self.device)),
                "talon_build_tree")
+
+    def prune_tree(self, tree: Tree, keep: int):
+        """``talon_prune_tree``: the final Top-N step of the static construction (Algorithm 1)."""
+        ts = tree.struct()
+        _check(_lib.talon_prune_tree(self._ctx, C.byref(ts), int(keep), _stream(self.device)), "talon_prune_tree")
 
     def tree_attention(self, tree: Tree, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_tokens, kv_stride_t,
                        kv_stride_h, max_prefix_len, sm_scale, out):
