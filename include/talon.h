@@ -275,6 +275,68 @@ talon_status talon_step(talon_ctx *ctx, const talon_tree *tree, int32_t B, const
                         int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
                         void *stream);
 
+/* Paged prefix cache (the layout serving systems keep for batches, which the paper's "Limitations"
+ * name as the open case; Section 5.3's loop is the same).  The cache is a pool of pages of
+ * TALON_PAGE_TOKENS tokens: token t of sequence b lives in page block_table[b, t / 128] at offset
+ * t % 128, i.e. at cache token page * 128 + offset of a [n_pages * 128, Hkv, Dh] array with the
+ * usual strides.  A page is one key tile of the attention kernel, so a tile never straddles pages.
+ *  block_table   device [B, table_stride] int32 page numbers; a sequence needs
+ *                ceil(prefix_len / 128) entries (talon_commit_paged: up to n_blocks[b])
+ *  n_pages       pages in the pool (bounds the tensor map)
+ * Otherwise as talon_tree_attention.  Query-group sizes that do not divide 128 return
+ * TALON_ERR_UNSUPPORTED here (the warp-MMA kernel reads contiguous blocks only). */
+#define TALON_PAGE_TOKENS 128
+talon_status talon_tree_attention_paged(talon_ctx *ctx, const talon_tree *tree, const void *q,
+                                        const void *k_pages, const void *v_pages, const void *k_tree,
+                                        const void *v_tree, const int32_t *block_table,
+                                        int32_t table_stride, int64_t n_pages, int64_t kv_stride_t,
+                                        int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale,
+                                        void *out, void *stream);
+
+/* talon_commit on a paged cache: the accepted path's K/V rows go to tokens prefix_len[b] + j of
+ * sequence b through the page table.
+ *  n_blocks  device [B]: pages the sequence owns (entries of its block_table row that are valid);
+ *            a sequence whose accepted tokens do not fit in them is left untouched and
+ *            TALON_ERR_CAPACITY is reported by talon_poll_status. */
+talon_status talon_commit_paged(talon_ctx *ctx, const talon_tree *tree, const int32_t *accept_len,
+                                const int32_t *accept_nodes, const int32_t *next_tok,
+                                const void *k_tree, const void *v_tree, void *k_pages, void *v_pages,
+                                const int32_t *block_table, int32_t table_stride,
+                                const int32_t *n_blocks, int64_t n_pages, int64_t kv_stride_t,
+                                int64_t kv_stride_h, int32_t *prefix_len, int32_t *root_tok,
+                                int64_t *counters, void *stream);
+
+/* Section 5.3's generation loop, n_steps draft-and-verify steps in one call: for every step the
+ * launches of talon_step followed by talon_commit, so that the accepted tokens' K/V join the
+ * prefix cache, prefix_len grows and the correction token is the next step's root, all on the
+ * device (the call only enqueues; a caller may capture it into one CUDA graph).  The stand-ins for
+ * the two model forwards are indexed by step: step s reads draft_logits + s * draft_step_stride,
+ * target_logits + s * target_step_stride, q + s * q_step_stride and k_tree / v_tree +
+ * s * kv_tree_step_stride (strides in elements), and writes accept_len / bonus_tok at
+ * + s * result_step_stride and accept_nodes at + s * result_step_stride * (D_max + 1) (a stride of 0
+ * keeps only the last step's).  root_tok, prefix_len, the cache and counters ([B, 3], as in
+ * talon_commit; required) are read and advanced in place.
+ *  max_prefix_len  bound on prefix_len[b] over ALL steps (the last step's prefix included) */
+talon_status talon_loop(talon_ctx *ctx, const talon_tree *tree, int32_t B, int32_t n_steps,
+                        int32_t *root_tok, int32_t *prefix_len, const float *draft_logits,
+                        int64_t draft_row_stride, int64_t draft_step_stride, int32_t n_layers,
+                        const void *q, int64_t q_step_stride, void *k_prefix, void *v_prefix,
+                        const void *k_tree, const void *v_tree, int64_t kv_tree_step_stride,
+                        const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
+                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len,
+                        float sm_scale, void *out, const float *target_logits,
+                        int64_t target_row_stride, int64_t target_step_stride, int32_t *target_tok,
+                        int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                        int64_t result_step_stride, int64_t *counters, void *stream);
+
+/* Section 5.3's figures from the counters talon_commit keeps (HOST copy of the [B, 3] array: N_p
+ * verification passes, N_q draft passes, L tokens produced), summed over the sequences: draft
+ * efficiency delta = N_q / N_p (Eq. 6), mean accepted tokens tau = L / N_p, and the wall-time
+ * speed-up R = tau / (1 + c * delta) (Eq. 7) for a draft pass that costs cost_ratio = c target
+ * passes.  Host arithmetic only; TALON_ERR_INVALID_ARG when no pass has been committed. */
+talon_status talon_loop_metrics(const int64_t *counters, int32_t B, double cost_ratio, double *delta,
+                                double *tau, double *speedup);
+
 /* The paper has no counterpart for this call: it exists for callers that cannot allocate.
  * talon_accept needs a context, and talon_create calls cudaMalloc.  Code that runs inside a
  * fixed memory pool, or in a part of a serving loop where allocating is not allowed (it

@@ -237,8 +237,27 @@ talon_status talon_tree_attention(talon_ctx *c, const talon_tree *t, const void 
     return TALON_ERR_INVALID_ARG;
   if (!(sm_scale == sm_scale)) return TALON_ERR_INVALID_ARG;
   return talon::launch_attention(c, t, q, k_prefix ? k_prefix : k_tree, v_prefix ? v_prefix : v_tree, k_tree,
-                                 v_tree, kv_start, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale,
-                                 out, (cudaStream_t)stream);
+                                 v_tree, kv_start, nullptr, 0, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len,
+                                 sm_scale, out, (cudaStream_t)stream);
+}
+
+talon_status talon_tree_attention_paged(talon_ctx *c, const talon_tree *t, const void *q, const void *k_pages,
+                                        const void *v_pages, const void *k_tree, const void *v_tree,
+                                        const int32_t *block_table, int32_t table_stride, int64_t n_pages,
+                                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len,
+                                        float sm_scale, void *out, void *stream) {
+  if (!c || !tree_complete(t) || !q || !k_tree || !v_tree || !block_table || !out) return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || max_prefix_len < 0 || n_pages < 0 || n_pages * TALON_PAGE_TOKENS > 0x7FFFFFFFll) return TALON_ERR_INVALID_ARG;
+  if (table_stride < (max_prefix_len + TALON_PAGE_TOKENS - 1) / TALON_PAGE_TOKENS) return TALON_ERR_INVALID_ARG;
+  if (max_prefix_len > 0 && (!k_pages || !v_pages || n_pages < 1)) return TALON_ERR_INVALID_ARG;
+  if ((kv_stride_t & 7) || (kv_stride_h & 7) || kv_stride_t < 0 || kv_stride_h < 0) return TALON_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(k_tree) || !aligned16(v_tree) ||
+      !aligned16(out))
+    return TALON_ERR_INVALID_ARG;
+  if (!(sm_scale == sm_scale)) return TALON_ERR_INVALID_ARG;
+  return talon::launch_attention(c, t, q, k_pages ? k_pages : k_tree, v_pages ? v_pages : v_tree, k_tree, v_tree,
+                                 nullptr, block_table, table_stride, n_pages * TALON_PAGE_TOKENS, kv_stride_t,
+                                 kv_stride_h, max_prefix_len, sm_scale, out, (cudaStream_t)stream);
 }
 
 talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
@@ -276,8 +295,80 @@ talon_status talon_commit(talon_ctx *c, const talon_tree *t, const int32_t *acce
   if (!aligned16(k_prefix) || !aligned16(v_prefix) || !aligned16(k_tree) || !aligned16(v_tree))
     return TALON_ERR_INVALID_ARG;
   return talon::launch_commit(c, t, accept_len, accept_nodes, next_tok, k_tree, v_tree, k_prefix, v_prefix, kv_start,
-                              kv_limit, kv_tokens, kv_stride_t, kv_stride_h, prefix_len, root_tok, counters,
-                              (cudaStream_t)stream);
+                              kv_limit, nullptr, 0, nullptr, kv_tokens, kv_stride_t, kv_stride_h, prefix_len, root_tok,
+                              counters, (cudaStream_t)stream);
+}
+
+talon_status talon_commit_paged(talon_ctx *c, const talon_tree *t, const int32_t *accept_len,
+                                const int32_t *accept_nodes, const int32_t *next_tok, const void *k_tree,
+                                const void *v_tree, void *k_pages, void *v_pages, const int32_t *block_table,
+                                int32_t table_stride, const int32_t *n_blocks, int64_t n_pages, int64_t kv_stride_t,
+                                int64_t kv_stride_h, int32_t *prefix_len, int32_t *root_tok, int64_t *counters,
+                                void *stream) {
+  if (!c || !tree_complete(t) || !accept_len || !accept_nodes || !next_tok || !k_tree || !v_tree || !k_pages ||
+      !v_pages || !block_table || !n_blocks || !prefix_len || !root_tok)
+    return TALON_ERR_INVALID_ARG;
+  if (c->B < 1 || n_pages < 1 || n_pages * TALON_PAGE_TOKENS > 0x7FFFFFFFll || table_stride < 1) return TALON_ERR_INVALID_ARG;
+  if ((kv_stride_t & 7) || (kv_stride_h & 7) || kv_stride_t < 0 || kv_stride_h < 0) return TALON_ERR_INVALID_ARG;
+  if (!aligned16(k_pages) || !aligned16(v_pages) || !aligned16(k_tree) || !aligned16(v_tree)) return TALON_ERR_INVALID_ARG;
+  return talon::launch_commit(c, t, accept_len, accept_nodes, next_tok, k_tree, v_tree, k_pages, v_pages, nullptr, nullptr,
+                              block_table, table_stride, n_blocks, n_pages * TALON_PAGE_TOKENS, kv_stride_t, kv_stride_h,
+                              prefix_len, root_tok, counters, (cudaStream_t)stream);
+}
+
+static talon_status step_enqueue(talon_ctx *c, const talon_tree *t, int32_t B, const int32_t *root_tok,
+                                 const int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
+                                 int32_t n_layers, const void *q, const void *k_prefix, const void *v_prefix,
+                                 const void *k_tree, const void *v_tree, const int64_t *kv_start, int64_t kv_tokens,
+                                 int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale,
+                                 void *out, const float *target_logits, int64_t target_row_stride,
+                                 int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                                 void *stream);
+
+talon_status talon_loop(talon_ctx *c, const talon_tree *t, int32_t B, int32_t n_steps, int32_t *root_tok,
+                        int32_t *prefix_len, const float *draft_logits, int64_t draft_row_stride,
+                        int64_t draft_step_stride, int32_t n_layers, const void *q, int64_t q_step_stride,
+                        void *k_prefix, void *v_prefix, const void *k_tree, const void *v_tree,
+                        int64_t kv_tree_step_stride, const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
+                        int64_t kv_stride_t, int64_t kv_stride_h, int32_t max_prefix_len, float sm_scale, void *out,
+                        const float *target_logits, int64_t target_row_stride, int64_t target_step_stride,
+                        int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                        int64_t result_step_stride, int64_t *counters, void *stream) {
+  if (!c || n_steps < 1 || !root_tok || !prefix_len || !counters) return TALON_ERR_INVALID_ARG;
+  if (n_layers < 0 || n_layers > c->p.max_depth) return TALON_ERR_INVALID_ARG;
+  if (draft_step_stride < 0 || q_step_stride < 0 || kv_tree_step_stride < 0 || target_step_stride < 0 ||
+      result_step_stride < 0 || (q_step_stride & 7) || (kv_tree_step_stride & 7) || (draft_step_stride & 3) ||
+      (target_step_stride & 3))
+    return TALON_ERR_INVALID_ARG;
+  const char *qb = static_cast<const char *>(q), *ktb = static_cast<const char *>(k_tree), *vtb = static_cast<const char *>(v_tree);
+  for (int s = 0; s < n_steps; ++s) {
+    // step s reads its own slice of the stand-ins for the two model forwards; the tree, the cache,
+    // the prefix lengths and the roots are the state the steps hand on to one another on the device
+    const void *qs = qb + 2 * q_step_stride * s, *kts = ktb + 2 * kv_tree_step_stride * s, *vts = vtb + 2 * kv_tree_step_stride * s;
+    int32_t *al = accept_len + result_step_stride * s, *an = accept_nodes + result_step_stride * (c->p.max_depth + 1) * s;
+    int32_t *bt = bonus_tok + result_step_stride * s;
+    talon_status r = step_enqueue(c, t, B, root_tok, prefix_len, draft_logits + draft_step_stride * s, draft_row_stride,
+                                  n_layers, qs, k_prefix, v_prefix, kts, vts, kv_start, kv_tokens, kv_stride_t, kv_stride_h,
+                                  max_prefix_len, sm_scale, out, target_logits + target_step_stride * s, target_row_stride,
+                                  target_tok, al, an, bt, stream);
+    if (r == TALON_OK)
+      r = talon_commit(c, t, al, an, bt, kts, vts, k_prefix, v_prefix, kv_start, kv_limit, kv_tokens, kv_stride_t,
+                       kv_stride_h, prefix_len, root_tok, counters, stream);
+    if (r != TALON_OK) return r;
+  }
+  return TALON_OK;
+}
+
+talon_status talon_loop_metrics(const int64_t *counters, int32_t B, double cost_ratio, double *delta, double *tau,
+                                double *speedup) {
+  if (!counters || B < 1 || !delta || !tau || !speedup || !(cost_ratio >= 0.0)) return TALON_ERR_INVALID_ARG;
+  long long n_p = 0, n_q = 0, len = 0;
+  for (int b = 0; b < B; ++b) { n_p += counters[3 * b]; n_q += counters[3 * b + 1]; len += counters[3 * b + 2]; }
+  if (n_p <= 0) return TALON_ERR_INVALID_ARG;
+  *delta = (double)n_q / (double)n_p;                  // Eq. 6: draft passes per verification pass
+  *tau = (double)len / (double)n_p;                    // mean accepted tokens per verification pass
+  *speedup = *tau / (1.0 + cost_ratio * *delta);       // Eq. 7
+  return TALON_OK;
 }
 
 talon_status talon_poll_status(talon_ctx *c, void *stream) {

@@ -344,7 +344,8 @@ talon_status attention_mma_setup() {
 }
 
 talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
-                              const void *kt, const void *vt, const int64_t *kv_start, int64_t kv_tokens,
+                              const void *kt, const void *vt, const int64_t *kv_start, const int32_t *block_table,
+                              int bt_stride, int64_t kv_tokens,
                               int64_t stride_t, int64_t stride_h, int max_prefix_len, float sm_scale, void *out,
                               cudaStream_t st) {
   AttnArgs a;
@@ -384,7 +385,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
     }
     while (sp > 1 && (size_t)a.m_blocks * c->B * a.Hkv * sp * AT_BM > c->attn_ml_elems) --sp;
     a.splits = sp;
-    talon_status r = launch_attention_tc(c, t, q, kp, vp, kt, vt, kv_start, stride_t, stride_h, kv_tokens,
+    talon_status r = launch_attention_tc(c, t, q, kp, vp, kt, vt, kv_start, block_table, bt_stride, stride_t, stride_h, kv_tokens,
                                          max_prefix_len, sm_scale, out, sp, a.m_blocks, st);
     if (r != TALON_OK) return r;
     if (sp > 1) {
@@ -398,6 +399,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
     return TALON_OK;
   }
 
+  if (block_table) return TALON_ERR_UNSUPPORTED;     // the warp-MMA kernel reads contiguous blocks only
   const int base = a.m_blocks * c->B * a.Hkv;
   const int max_tiles = (max_prefix_len + AT_BN - 1) / AT_BN + (a.N + AT_BN - 1) / AT_BN;
   int splits = 1;

@@ -52,6 +52,8 @@ enum { B_Q = 0, B_KFULL = 1, B_VFULL = 3, B_KEMPTY = 5, B_VEMPTY = 7, B_SFULL = 
 
 struct TcArgs {
   const int64_t *kv_start;
+  const int32_t *block_table;  // paged prefix: [B, bt_stride] page numbers (null: contiguous blocks at kv_start)
+  int bt_stride;
   const int32_t *prefix_len, *n_nodes;
   const unsigned long long *mask;
   int B, N, W, Hq, Hkv, g;
@@ -271,7 +273,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         for (int h = 0; h < 2; ++h)
           tma_load_4d(q_smem + i * TC_TILE_BYTES + h * TC_HALF_BYTES, &map_q, bar(B_Q), h * 64, kvh * a.g,
                       (mpair * 2 + i) * nodes_per_tile, b);
-      const long long tok0 = a.kv_start[b];
+      // first cache token of prefix tile tg: a page of TC_BN tokens from the table, or the
+      // sequence's contiguous block
+      const long long tok0 = a.block_table ? 0ll : a.kv_start[b];
+      auto tile_tok = [&](int tg) {
+        return a.block_table ? (long long)a.block_table[(size_t)b * a.bt_stride + tg] * TC_BN : tok0 + (long long)tg * TC_BN;
+      };
       bool ok = true;
       for (int it = 0; it < nt && ok; ++it) {
         const int s = it % TC_STAGES;
@@ -282,7 +289,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         mbar_expect_tx(bar(B_KFULL + s), TC_TILE_BYTES);
         for (int h = 0; h < 2; ++h) {
           const uint32_t dst = k_smem + s * TC_TILE_BYTES + h * TC_HALF_BYTES;
-          if (tg < nP) tma_load_3d(dst, &map_kp, bar(B_KFULL + s), h * 64, kvh, (int)(tok0 + (long long)tg * TC_BN));
+          if (tg < nP) tma_load_3d(dst, &map_kp, bar(B_KFULL + s), h * 64, kvh, (int)tile_tok(tg));
           else tma_load_4d(dst, &map_kt, bar(B_KFULL + s), h * 64, kvh, (tg - nP) * TC_BN, b);
         }
         ok = mbar_wait(bar(B_VEMPTY + s), par, abort_flag);
@@ -290,7 +297,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         mbar_expect_tx(bar(B_VFULL + s), TC_TILE_BYTES);
         for (int h = 0; h < 2; ++h) {
           const uint32_t dst = v_smem + s * TC_TILE_BYTES + h * TC_HALF_BYTES;
-          if (tg < nP) tma_load_3d(dst, &map_vp, bar(B_VFULL + s), h * 64, kvh, (int)(tok0 + (long long)tg * TC_BN));
+          if (tg < nP) tma_load_3d(dst, &map_vp, bar(B_VFULL + s), h * 64, kvh, (int)tile_tok(tg));
           else tma_load_4d(dst, &map_vt, bar(B_VFULL + s), h * 64, kvh, (tg - nP) * TC_BN, b);
         }
       }
@@ -599,7 +606,8 @@ talon_status attention_tc_setup() {
 }
 
 talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
-                                 const void *kt, const void *vt, const int64_t *kv_start, int64_t stride_t,
+                                 const void *kt, const void *vt, const int64_t *kv_start, const int32_t *block_table,
+                                 int bt_stride, int64_t stride_t,
                                  int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
                                  int splits, int m_blocks, cudaStream_t st) {
   const int N = c->p.budget, Hq = c->p.n_q_heads, Hkv = c->p.n_kv_heads, g = Hq / Hkv, B = c->B;
@@ -623,7 +631,8 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
     if (!encode_bf16(&mkt, kt, 4, dims, str, box) || !encode_bf16(&mvt, vt, 4, dims, str, box)) return TALON_ERR_CUDA;
   }
   TcArgs a;
-  a.kv_start = kv_start; a.prefix_len = c->d_prefix_len; a.n_nodes = t->n_nodes;
+  a.kv_start = kv_start; a.block_table = block_table; a.bt_stride = bt_stride;
+  a.prefix_len = c->d_prefix_len; a.n_nodes = t->n_nodes;
   a.mask = (const unsigned long long *)t->mask;
   a.B = B; a.N = N; a.W = c->W; a.Hq = Hq; a.Hkv = Hkv; a.g = g;
   a.scale_log2 = sm_scale * 1.4426950408889634f;

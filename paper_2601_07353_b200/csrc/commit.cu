@@ -17,6 +17,8 @@ namespace talon {
 
 namespace {
 
+constexpr int COMMIT_PAGE = 128;          // tokens per page of a paged cache (one key tile of the attention)
+
 struct CommitArgs {
   talon_tree t;
   int lo_stride;
@@ -25,6 +27,8 @@ struct CommitArgs {
   const uint4 *k_tree, *v_tree;       // [B, N, Hkv, Dh] bf16
   uint4 *k_prefix, *v_prefix;
   const int64_t *kv_start, *kv_limit;
+  const int32_t *block_table, *n_blocks;   // paged cache: [B, bt_stride] page numbers, [B] pages a sequence owns
+  int bt_stride;
   int64_t kv_tokens, stride_t, stride_h;   // elements
   int32_t *prefix_len, *root_tok;
   int64_t *counters;                  // [B, 3] or null
@@ -38,7 +42,16 @@ __device__ __forceinline__ int64_t block_end(const CommitArgs &a, int b) {
 }
 
 __device__ __forceinline__ bool fits(const CommitArgs &a, int b, int len) {
-  return len >= 0 && len <= a.max_depth && a.kv_start[b] + a.prefix_len[b] + len + 1 <= block_end(a, b);
+  if (len < 0 || len > a.max_depth) return false;
+  if (a.block_table) return (int64_t)a.prefix_len[b] + len + 1 <= (int64_t)a.n_blocks[b] * COMMIT_PAGE;
+  return a.kv_start[b] + a.prefix_len[b] + len + 1 <= block_end(a, b);
+}
+
+// cache token that holds token `pos` of sequence b
+__device__ __forceinline__ int64_t cache_token(const CommitArgs &a, int b, int pos) {
+  if (a.block_table)
+    return (int64_t)a.block_table[(size_t)b * a.bt_stride + pos / COMMIT_PAGE] * COMMIT_PAGE + pos % COMMIT_PAGE;
+  return a.kv_start[b] + pos;
 }
 
 __global__ void commit_gather_kernel(CommitArgs a) {
@@ -50,7 +63,7 @@ __global__ void commit_gather_kernel(CommitArgs a) {
   if (node < 0 || node >= a.N) return;                      // a malformed path never indexes outside the tree
   const int vec_per_head = a.head_dim / 8;                  // 16-byte units per head row
   const int vecs = a.n_kv_heads * vec_per_head;
-  const int64_t tok = a.kv_start[b] + a.prefix_len[b] + j;
+  const int64_t tok = cache_token(a, b, a.prefix_len[b] + j);
   const size_t src = ((size_t)b * a.N + node) * vecs;
   for (int i = threadIdx.x; i < 2 * vecs; i += blockDim.x) {
     const int which = i >= vecs, r = which ? i - vecs : i;
@@ -87,9 +100,9 @@ __global__ void commit_update_kernel(CommitArgs a) {
 
 talon_status launch_commit(talon_ctx *c, const talon_tree *t, const int32_t *accept_len, const int32_t *accept_nodes,
                            const int32_t *next_tok, const void *k_tree, const void *v_tree, void *k_prefix,
-                           void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
-                           int64_t stride_t, int64_t stride_h, int32_t *prefix_len, int32_t *root_tok,
-                           int64_t *counters, cudaStream_t st) {
+                           void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, const int32_t *block_table,
+                           int bt_stride, const int32_t *n_blocks, int64_t kv_tokens, int64_t stride_t, int64_t stride_h,
+                           int32_t *prefix_len, int32_t *root_tok, int64_t *counters, cudaStream_t st) {
   CommitArgs a;
   a.t = *t; a.lo_stride = c->p.max_depth + 2;
   a.B = c->B; a.N = c->p.budget; a.max_depth = c->p.max_depth; a.layers_run = c->layers_run;
@@ -97,7 +110,8 @@ talon_status launch_commit(talon_ctx *c, const talon_tree *t, const int32_t *acc
   a.accept_len = accept_len; a.accept_nodes = accept_nodes; a.next_tok = next_tok;
   a.k_tree = static_cast<const uint4 *>(k_tree); a.v_tree = static_cast<const uint4 *>(v_tree);
   a.k_prefix = static_cast<uint4 *>(k_prefix); a.v_prefix = static_cast<uint4 *>(v_prefix);
-  a.kv_start = kv_start; a.kv_limit = kv_limit; a.kv_tokens = kv_tokens; a.stride_t = stride_t; a.stride_h = stride_h;
+  a.kv_start = kv_start; a.kv_limit = kv_limit; a.block_table = block_table; a.n_blocks = n_blocks; a.bt_stride = bt_stride;
+  a.kv_tokens = kv_tokens; a.stride_t = stride_t; a.stride_h = stride_h;
   a.prefix_len = prefix_len; a.root_tok = root_tok; a.counters = counters; a.status = c->d_status;
   {
     LaunchTimer lt(c, TALON_K_COMMIT, st);

@@ -204,12 +204,13 @@ talon_status launch_build(talon_ctx *c, const talon_tree *t, uint8_t *dense, cud
 talon_status launch_prune(talon_ctx *c, const talon_tree *t, int keep, cudaStream_t st);
 talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, const void *kp,
                               const void *vp, const void *kt, const void *vt,
-                              const int64_t *kv_start, int64_t kv_tokens, int64_t stride_t, int64_t stride_h,
+                              const int64_t *kv_start, const int32_t *block_table, int bt_stride, int64_t kv_tokens,
+                              int64_t stride_t, int64_t stride_h,
                               int max_prefix_len, float sm_scale, void *out, cudaStream_t st);
 bool attention_tc_supported(const talon_ctx *c, int64_t stride_t, int64_t stride_h, float sm_scale);
 talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
-                                 const void *kt, const void *vt, const int64_t *kv_start, int64_t stride_t,
-                                 int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
+                                 const void *kt, const void *vt, const int64_t *kv_start, const int32_t *block_table,
+                                 int bt_stride, int64_t stride_t, int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
                                  int splits, int m_blocks, cudaStream_t st);
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
@@ -219,9 +220,9 @@ talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float
                                   int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, cudaStream_t st);
 talon_status launch_commit(talon_ctx *c, const talon_tree *t, const int32_t *accept_len, const int32_t *accept_nodes,
                            const int32_t *next_tok, const void *k_tree, const void *v_tree, void *k_prefix,
-                           void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, int64_t kv_tokens,
-                           int64_t stride_t, int64_t stride_h, int32_t *prefix_len, int32_t *root_tok,
-                           int64_t *counters, cudaStream_t st);
+                           void *v_prefix, const int64_t *kv_start, const int64_t *kv_limit, const int32_t *block_table,
+                           int bt_stride, const int32_t *n_blocks, int64_t kv_tokens, int64_t stride_t, int64_t stride_h,
+                           int32_t *prefix_len, int32_t *root_tok, int64_t *counters, cudaStream_t st);
 size_t attention_workspace_elems(const talon_ctx *c, size_t *ml_elems);
 talon_status expand_fused_setup(talon_ctx *c);
 talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float *logits, int64_t row_stride,

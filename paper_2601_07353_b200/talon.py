@@ -46,6 +46,11 @@ _lib.talon_expand_layer.argtypes = [_vp, _TP, _vp, _i64, _i32, _i32, _vp]
 _lib.talon_layers_run.argtypes = [_vp]
 _lib.talon_build_tree.argtypes = [_vp, _TP, _vp, _vp]
 _lib.talon_prune_tree.argtypes = [_vp, _TP, _i32, _vp]
+_lib.talon_tree_attention_paged.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
+_lib.talon_commit_paged.argtypes = [_vp, _TP] + [_vp] * 8 + [_i32, _vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]
+_lib.talon_loop.argtypes = ([_vp, _TP, _i32, _i32, _vp, _vp, _vp, _i64, _i64, _i32, _vp, _i64, _vp, _vp, _vp, _vp, _i64, _vp, _vp,
+                            _i64, _i64, _i64, _i32, _f32, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp, _i64, _vp, _vp])
+_lib.talon_loop_metrics.argtypes = [_vp, _i32, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
 _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_accept_sample.argtypes = [_vp, _TP, _vp, _i64, C.c_double, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -67,7 +72,8 @@ _lib.talon_status_string.restype = C.c_char_p
 for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
            "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
-           "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit", "talon_prune_tree"):
+           "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit", "talon_prune_tree",
+           "talon_tree_attention_paged", "talon_commit_paged", "talon_loop", "talon_loop_metrics"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
@@ -75,7 +81,9 @@ EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer"
             "talon_step_host", "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
             "talon_kernel_name",
             "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample",
-            "talon_commit", "talon_prune_tree"]
+            "talon_commit", "talon_prune_tree", "talon_tree_attention_paged", "talon_commit_paged", "talon_loop",
+            "talon_loop_metrics"]
+PAGE_TOKENS = 128
 NOALLOC_MAX_ROWS = 8192
 N_KERNELS = 11
 KERNEL_NAMES = [_lib.talon_kernel_name(i).decode() for i in range(N_KERNELS)]
@@ -101,16 +109,14 @@ def _stream(device) -> C.c_void_p:
 
 
 def loop_metrics(counters: torch.Tensor, cost_ratio: float) -> dict:
-    """Section 5.3's figures from the counters ``talon_commit`` keeps ([B, 3] int64: verification
-    passes N_p, draft passes N_q, tokens produced L), summed over the sequences: draft efficiency
-    delta = N_q / N_p, mean accepted tokens tau = L / N_p and the wall-time speed-up
-    R = tau / (1 + c delta) for a draft pass that costs ``cost_ratio`` = c target passes."""
-    n_p, n_q, length = (int(x) for x in counters.sum(dim=0).tolist())
-    if n_p <= 0:
-        raise ValueError("no verification pass has been committed yet")
-    delta, tau = n_q / n_p, length / n_p
-    return {"n_p": n_p, "n_q": n_q, "tokens": length, "delta": delta, "tau": tau,
-            "speedup": tau / (1.0 + cost_ratio * delta)}
+    """``talon_loop_metrics``: Section 5.3's delta, tau and speed-up from the counters ``talon_commit``
+    keeps ([B, 3] int64).  The arithmetic is the library's; this only copies the counters to the host."""
+    host = counters.detach().to("cpu", torch.int64).contiguous()
+    d, t, r = C.c_double(), C.c_double(), C.c_double()
+    _check(_lib.talon_loop_metrics(C.c_void_p(host.data_ptr()), host.shape[0], float(cost_ratio), C.byref(d), C.byref(t),
+                                   C.byref(r)), "talon_loop_metrics")
+    n_p, n_q, length = (int(x) for x in host.sum(dim=0).tolist())
+    return {"n_p": n_p, "n_q": n_q, "tokens": length, "delta": d.value, "tau": t.value, "speedup": r.value}
 
 
 def target_argmax_noalloc(target_logits: torch.Tensor, target_tok: torch.Tensor) -> None:
@@ -239,6 +245,39 @@ class Talon:
                                  _ptr(k_tree), _ptr(v_tree), _ptr(k_prefix), _ptr(v_prefix), _ptr(kv_start),
                                  _ptr(kv_limit), kv_tokens, kv_stride_t, kv_stride_h, _ptr(prefix_len), _ptr(root_tok),
                                  _ptr(counters), _stream(self.device)), "talon_commit")
+
+    def tree_attention_paged(self, tree: Tree, q, k_pages, v_pages, k_tree, v_tree, block_table, n_pages, kv_stride_t,
+                             kv_stride_h, max_prefix_len, sm_scale, out):
+        ts = tree.struct()
+        _check(_lib.talon_tree_attention_paged(self._ctx, C.byref(ts), _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(k_tree),
+                                               _ptr(v_tree), _ptr(block_table), block_table.stride(0), n_pages, kv_stride_t,
+                                               kv_stride_h, max_prefix_len, sm_scale, _ptr(out), _stream(self.device)),
+               "talon_tree_attention_paged")
+
+    def commit_paged(self, tree: Tree, accept_len, accept_nodes, next_tok, k_tree, v_tree, k_pages, v_pages, block_table,
+                     n_blocks, n_pages, kv_stride_t, kv_stride_h, prefix_len, root_tok, counters=None):
+        ts = tree.struct()
+        _check(_lib.talon_commit_paged(self._ctx, C.byref(ts), _ptr(accept_len), _ptr(accept_nodes), _ptr(next_tok),
+                                       _ptr(k_tree), _ptr(v_tree), _ptr(k_pages), _ptr(v_pages), _ptr(block_table),
+                                       block_table.stride(0), _ptr(n_blocks), n_pages, kv_stride_t, kv_stride_h,
+                                       _ptr(prefix_len), _ptr(root_tok), _ptr(counters), _stream(self.device)),
+               "talon_commit_paged")
+
+    def loop(self, tree: Tree, n_steps, root_tok, prefix_len, draft, n_layers, q, k_prefix, v_prefix, k_tree, v_tree,
+             kv_start, kv_limit, kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, out, target, target_tok,
+             accept_len, accept_nodes, bonus_tok, counters, keep_results: bool = True):
+        """``talon_loop``: ``n_steps`` draft-and-verify steps with the commit between them.  ``draft`` and
+        ``target`` are [S, B, N, V]; ``q``, ``k_tree``, ``v_tree`` [S, B, N, H, Dh]; with ``keep_results`` the
+        result arrays are [S, B(, D_max + 1)], else the last step's."""
+        ts = tree.struct()
+        B = root_tok.shape[0]
+        _check(_lib.talon_loop(self._ctx, C.byref(ts), B, n_steps, _ptr(root_tok), _ptr(prefix_len), _ptr(draft),
+                               draft.stride(-2), draft.stride(0), n_layers, _ptr(q), q.stride(0), _ptr(k_prefix),
+                               _ptr(v_prefix), _ptr(k_tree), _ptr(v_tree), k_tree.stride(0), _ptr(kv_start), _ptr(kv_limit),
+                               kv_tokens, kv_stride_t, kv_stride_h, max_prefix_len, sm_scale, _ptr(out), _ptr(target),
+                               target.stride(-2), target.stride(0), _ptr(target_tok), _ptr(accept_len), _ptr(accept_nodes),
+                               _ptr(bonus_tok), B if keep_results else 0, _ptr(counters), _stream(self.device)),
+               "talon_loop")
 
     def poll_status(self) -> int:
         return _lib.talon_poll_status(self._ctx, _stream(self.device))

@@ -81,9 +81,12 @@ def logit_rows(B: int, N: int, V: int, row_pad: int, dev) -> torch.Tensor:
 
 def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAULT_SEED,
                    seq_ids: Optional[Sequence[int]] = None, with_verify: bool = True, row_pad: int = 0,
-                   prefix_lens: Optional[Sequence[int]] = None, host_inputs: bool = False) -> Workload:
+                   prefix_lens: Optional[Sequence[int]] = None, host_inputs: bool = False,
+                   root_tokens: Optional[Sequence[int]] = None) -> Workload:
     """``row_pad`` widens the logit rows' stride (NaN padding); ``prefix_lens`` overrides the hashed
     prefix lengths of the sequences (the generated K/V of a sequence are cut to that length);
+    ``root_tokens`` overrides the hashed root tokens (a later step of a generation loop starts from
+    the previous step's correction token);
     ``host_inputs`` generates every input with NumPy on the host and uploads it (bit-identical to
     the device generator), so that the only kernels the GPU runs are the library's."""
     dev = talon.device
@@ -92,7 +95,9 @@ def build_workload(cfg: synth.TalonConfig, talon: Talon, seed: int = synth.DEFAU
     seq_ids = list(range(cfg.batch)) if seq_ids is None else list(seq_ids)
     B, N, V = len(seq_ids), cfg.budget, cfg.vocab
     i32 = dict(dtype=torch.int32, device=dev)
-    root = torch.tensor([synth.root_token(cfg, seed, s) for s in seq_ids], **i32)
+    roots = [synth.root_token(cfg, seed, s) for s in seq_ids] if root_tokens is None else [int(x) for x in root_tokens]
+    assert len(roots) == B
+    root = torch.tensor(roots, **i32)
     plens = [synth.prefix_len(cfg, seed, s) for s in seq_ids] if prefix_lens is None else [int(x) for x in prefix_lens]
     assert len(plens) == B
     prefix_len = torch.tensor(plens, **i32)
