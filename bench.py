@@ -54,6 +54,7 @@ MIN_REGION_S = 0.5               # a timed region shorter than this is repeated
 KERNEL_REPLAYS = 24              # back-to-back replays per kernel-alone measurement (at least 20)
 HEADLINE = "longctx"
 SUB_CONFIGS = ["tiny", "llama8b", "llama8b_batched", "qwen32b"]
+LOOP_CONFIG = "llama8b"          # the workload the multi-step generation loop is run on as an extra
 ORACLE_PREFIX_SAMPLE = 4096      # prefix tokens the oracle's attention is timed on when the prefix is longer
 DTYPE = "f32 logits, f64 path scores, bf16 attention (f32 accumulate)"
 
@@ -383,6 +384,71 @@ def kernel_pass(t, cfg, sets, stream):
     return out, launches, replays
 
 
+def generation_loop_extra(t, cfg, args, dev, steps: int = 4):
+    """Section 5.3's loop as an extra: ``steps`` draft-and-verify steps with the commit between them as
+    ONE ``talon_loop`` call captured in one CUDA graph; delta, tau and R from the library's counters.
+    The steps' inputs are built one after the other (a step starts from its predecessor's correction
+    token and prefix length), then the whole loop is replayed from the same start."""
+    import torch
+    from paper_2601_07353_b200 import synth, talon, workload
+    B, N, D, Hq, Hkv, Dh = cfg.batch, cfg.budget, cfg.max_depth, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    seqs = list(range(B))
+    scale = 1.0 / math.sqrt(Dh)
+    room = steps * (D + 1)
+    lens = [synth.prefix_len(cfg, args.seed, s) for s in seqs]
+    roots = [synth.root_token(cfg, args.seed, s) for s in seqs]
+    blocks = [L + room for L in lens]
+    starts = np.concatenate([[0], np.cumsum(blocks)[:-1]]).astype(np.int64)
+    total = int(starts[-1] + blocks[-1])
+    i64 = lambda x: torch.tensor(np.asarray(x), dtype=torch.int64, device=dev)
+    kv_start, kv_limit = i64(starts), i64(starts + np.asarray(blocks, np.int64))
+    kc = torch.zeros(total, Hkv, Dh, dtype=torch.bfloat16, device=dev)
+    vc = torch.zeros(total, Hkv, Dh, dtype=torch.bfloat16, device=dev)
+    plen = torch.tensor(lens, dtype=torch.int32, device=dev)
+    root = torch.tensor(roots, dtype=torch.int32, device=dev)
+    counters = torch.zeros(B, 3, dtype=torch.int64, device=dev)
+    built = []
+    for s in range(steps):
+        wl = workload.build_workload(cfg, t, args.seed + 1000 + s, seqs, prefix_lens=plen.cpu().tolist(),
+                                     root_tokens=root.cpu().tolist())
+        if s == 0:
+            ws = wl.kv_start.cpu().numpy()
+            for b in range(B):
+                kc[starts[b]:starts[b] + lens[b]] = wl.k_prefix[int(ws[b]):int(ws[b]) + lens[b]]
+                vc[starts[b]:starts[b] + lens[b]] = wl.v_prefix[int(ws[b]):int(ws[b]) + lens[b]]
+        t.reset(wl.tree, root, plen)
+        for _ in range(D):
+            t.expand_layer(wl.tree, wl.draft)
+        t.build_tree(wl.tree)
+        t.tree_attention(wl.tree, wl.q, kc, vc, wl.k_tree, wl.v_tree, kv_start, total, Hkv * Dh, Dh, int(plen.max()), scale, wl.out)
+        t.accept(wl.tree, wl.target, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok)
+        t.commit(wl.tree, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.k_tree, wl.v_tree, kc, vc, kv_start, kv_limit,
+                 total, Hkv * Dh, Dh, plen, root, counters)
+        built.append(wl)
+    assert t.poll_status() == talon.OK
+    draft = torch.stack([w.draft for w in built]); target = torch.stack([w.target for w in built])
+    q = torch.stack([w.q for w in built]); kt = torch.stack([w.k_tree for w in built]); vt = torch.stack([w.v_tree for w in built])
+    tree, out = built[0].tree, built[0].out
+    al = torch.zeros(steps, B, dtype=torch.int32, device=dev); an = torch.zeros(steps, B, D + 1, dtype=torch.int32, device=dev)
+    bo = torch.zeros(steps, B, dtype=torch.int32, device=dev); tt = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    plen0, root0 = torch.tensor(lens, dtype=torch.int32, device=dev), torch.tensor(roots, dtype=torch.int32, device=dev)
+    side = torch.cuda.Stream(dev)
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            plen.copy_(plen0); root.copy_(root0); counters.zero_()       # every replay starts from the same state
+            t.loop(tree, steps, root, plen, draft, D, q, kc, vc, kt, vt, kv_start, kv_limit, total, Hkv * Dh, Dh,
+                   max(lens) + room, scale, out, target, tt, al, an, bo, counters)
+        ms = time_replays([g], KERNEL_REPLAYS)
+    assert t.poll_status() == talon.OK
+    m5, m10 = talon.loop_metrics(counters, 0.05), talon.loop_metrics(counters, 0.10)
+    return {"steps_per_call": steps, "ms_per_call": ms, "value": steps / (ms * 1e-3), "unit": UNIT,
+            "delta": m5["delta"], "tau": m5["tau"], "speedup_R_at_c_0.05": m5["speedup"], "speedup_R_at_c_0.10": m10["speedup"],
+            "note": "talon_loop (step + commit per step) captured in one CUDA graph; delta = N_q/N_p, tau = L/N_p, "
+                    "R = tau/(1 + c delta) from the library's counters; the acceptance statistics are those of the synthetic "
+                    "target logits, not of a model"}
+
+
 def measure(cfg, args, info, dev, dev_index, peaks, headline: bool, sampler=None):
     """Builds the workload of ``cfg`` and measures it.  Returns the fields of a result line."""
     import torch
@@ -494,6 +560,12 @@ def measure(cfg, args, info, dev, dev_index, peaks, headline: bool, sampler=None
                      "frac": kd["frac_of_bf16_sustained"], "flop_per_byte": intensity, "ridge_flop_per_byte": ridge})
     res["roofline"] = roof
 
+    if cfg.name == LOOP_CONFIG and not args.no_loop:
+        try:
+            res["generation_loop"] = generation_loop_extra(t, cfg, args, dev)
+        except Exception as e:                           # an extra, never the headline
+            res["generation_loop"] = {"error": str(e).splitlines()[0][:200]}
+            torch.cuda.synchronize()
     if not headline:
         t.close()
         del sets
@@ -635,7 +707,8 @@ def run_talon(args):
         r.pop("timed_wall")
         others[name] = {"workload": workload_text(synth.CONFIGS[name]),
                         **{k: r[k] for k in ("value", "ms_per_step", "steps", "repeats", "spread", "roofline", "kernels",
-                                             "kernels_sum_over_step", "tree_shapes", "input_sets", "gpu_launches")}}
+                                             "kernels_sum_over_step", "tree_shapes", "input_sets", "gpu_launches")},
+                        **({"generation_loop": r["generation_loop"]} if "generation_loop" in r else {})}
     if sampler is not None:
         sampler.stop()
 
@@ -655,6 +728,7 @@ def run_talon(args):
             "graph_replay": head.get("graph_replay"), "kernels": head["kernels"], "kernel_timing": head["kernel_timing"],
             "kernels_sum_over_step": head["kernels_sum_over_step"], "sampling_verify": head.get("sampling_verify"),
             "tree_shapes": head["tree_shapes"], "sequence_steps_per_s": head["sequence_steps_per_s"],
+            "generation_loop": head.get("generation_loop"),
             "configs": others,
         }
         print(json.dumps(line))
@@ -744,6 +818,7 @@ def main(argv=None):
     ap.add_argument("--no-sampling", action="store_true", help="skip the sampling-verification extra")
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-repeat", action="store_true", help="time the K steps once, however short")
+    ap.add_argument("--no-loop", action="store_true", help="skip the multi-step generation-loop extra")
     ap.add_argument("--zipf-micro", action="store_true",
                     help="instead of the step benchmark: single-layer expansion latency on Zipf rows")
     args = ap.parse_args(argv)
