@@ -44,7 +44,7 @@ typedef unsigned long long u64;
 constexpr int XS_WTILE = 512;                 // floats a warp takes per step: 16 per lane, one 2 KB copy
 constexpr int XS_RING = 3;                    // copies in flight per warp
 constexpr int XS_BUF = FX_QCAP;               // keys a warp's candidate buffer holds
-constexpr int XS_POOL = 512;                  // keys the CTA pool holds
+constexpr int XS_POOL = 384;                  // keys the CTA pool holds
 constexpr int XS_TWO_LEVEL = EXP_WARPS;       // frontiers wider than this merge their rows all over the grid
 static_assert(XS_WTILE * EXP_WARPS == EXP_TILE, "a CTA step is eight warp tiles");
 static_assert(XS_BUF >= 64 && XS_POOL >= EXP_WARPS * 32, "buffers must hold a cut-back list plus one ballot");
@@ -55,7 +55,7 @@ struct FusedArgs {
   int rows_per_seq, layout;
   talon_tree t;
   int lo_stride;
-  int B, N, W, V, d, k, key_stride, max_split;
+  int B, N, W, V, d, k, key_stride, max_split, base_offset;
   int root_topk, init_layers;
   double log_mu;
   u64 *part_keys;          // [items, key_stride]  per-chunk top-k, descending
@@ -368,9 +368,9 @@ __device__ __forceinline__ void cut_back(u64 *buf, int ke, WarpStream &w, int la
 // Raises the warp's threshold from what it has seen so far (see the header of this file).
 // s_wtop[w] holds warp w's (share_pos + 1)-th largest lane maximum, s_wmax[w] its largest.
 __device__ __forceinline__ void refresh_threshold(WarpStream &w, int ke, int share_pos, bool gated, float ln_mu,
-                                                  float *s_wtop, float *s_wmax, int lane, int warp) {
+                                                  float *s_wtop, float *s_wmax, int lane, int warp, bool exact) {
   float cand, wmax, mine;
-  if (share_pos == 0) {
+  if (share_pos == 0 && !exact) {
     // ke <= 8: the eight 4-lane groups hold eight different elements at least as large as the
     // smallest group maximum; the warp maximum is what the other warps get to see
     float g = fmaxf(w.m_t, __shfl_xor_sync(FULL, w.m_t, 1));
@@ -425,24 +425,27 @@ __device__ __forceinline__ void collect_tile(const float *slot, const float (&v)
     if (lane >= o) inc += t;
   }
   const int total = __shfl_sync(FULL, inc, 31);
-  if (w.thr_key == 0ull && w.cnt + total <= XS_BUF) {
-    // the usual case: a handful of elements in a few lanes; each lane fetches its own from the slot
+  if (w.cnt + total <= XS_BUF) {
+    // the usual case: a handful of elements in a few lanes; each lane fetches its own from the
+    // slot.  After a cut-back only keys above the buffer's k-th count: the others leave an empty
+    // slot (key 0), which every reader of the buffer skips.
     int pos = w.cnt + inc - c;
     while (mm) {
       const int i = __ffs(mm) - 1;
       mm &= mm - 1u;
       const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
-      buf[pos++] = cand_key(slot[e], (uint32_t)(tok_tile + e));
+      const u64 key = cand_key(slot[e], (uint32_t)(tok_tile + e));
+      buf[pos++] = key > w.thr_key ? key : 0ull;
     }
     w.cnt += total;
     __syncwarp();
     if (w.cnt > XS_BUF - 32) cut_back(buf, ke, w, lane);
     return;
   }
-  // After a cut-back only keys above the buffer's k-th enter, and more may arrive than the buffer
-  // holds (equal logits, a sorted row, a cold threshold): take the tile one register slot at a
-  // time, cutting back whenever a ballot's worth might not fit.
-  if (w.cnt + total > XS_BUF) cut_back(buf, ke, w, lane);
+  // More than the buffer holds (equal logits, a sorted row, a cold threshold): cut the buffer
+  // back, then take the tile one register slot at a time, cutting back whenever a ballot's worth
+  // might not fit.
+  cut_back(buf, ke, w, lane);
 #pragma unroll 1
   for (int i = 0; i < 16; ++i) {
     const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
@@ -691,7 +694,6 @@ expand_fused_kernel(FusedArgs a) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ u64 s_buf[EXP_WARPS][XS_BUF];          // per-warp buffers of keys that reached the threshold
   __shared__ u64 s_pool[XS_POOL];                   // the chunk's candidates, all warps
-  __shared__ int s_base[MAX_BATCH + 1];
   __shared__ int s_warp[EXP_WARPS];
   __shared__ float s_m[EXP_WARPS], s_s[EXP_WARPS];
   __shared__ __align__(8) u64 s_bar[EXP_WARPS][XS_RING];   // "tile landed" barriers, per warp
@@ -717,6 +719,8 @@ expand_fused_kernel(FusedArgs a) {
   // ---- frontier geometry (from layer_off[d], layer_off[d + 1]: never written by this launch) ----
   Frontier fr;
   fr.in_regs = a.B <= 32;
+  // batches above 32 keep their frontier bases behind the ring (the launch adds the room)
+  int *s_base = reinterpret_cast<int *>(smem_raw + a.base_offset);
   fr.s_base = s_base;
   fr.base_l = fr.f_l = fr.lo_l = 0;
   if (fr.in_regs) {
@@ -843,17 +847,19 @@ expand_fused_kernel(FusedArgs a) {
         unpack_f32x2(add_f32x2(acc0, acc1), s0, s1);
         w.s_t += s0 + s1;
       }
-      refreshed = (t & (t + 1)) == 0;            // after tiles 1, 2, 4, 8, ... of the slice
-      if (refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp);
-      if (__ballot_sync(FULL, bm >= w.thr_f) != 0u)
+      refreshed = t < 4 || (t & 3) == 3;         // the threshold is cheap to refresh and pays early
+      // (the first tile has nothing but its own lane maxima to go by: their exact ke-th largest)
+      if (refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp, t == 0);
+      if (__ballot_sync(FULL, bm >= w.thr_f) != 0u) {
         collect_tile(ring + sl * XS_WTILE, v, base, ke, buf, w, lane);
+        __syncwarp();
+      }
       // Every lane's loads from the slot have delivered their data (the vote needs every lane's
       // maximum, and what the collection read has gone into the buffer): the slot can take the
       // tile XS_RING ahead.
-      __syncwarp();
       if (lane == 0 && t + XS_RING < nt) issue(t + XS_RING, wt - 1 + XS_RING);
     }
-    if (nt > 0 && !refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp);
+    if (nt > 0 && !refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp, false);
 
     // ---- the warp's survivors -> the CTA pool; its normaliser -> shared memory ----
     {
@@ -862,7 +868,7 @@ expand_fused_kernel(FusedArgs a) {
       const int n = w.cnt;
       for (int i = lane; i < n; i += 32) {
         const u64 key = buf[i];
-        if (key_logit(key) >= w.thr_f) {
+        if (key != 0ull && key_logit(key) >= w.thr_f) {
           const int pos = atomicAdd(&s_pool_n, 1);
           if (pos < XS_POOL) s_pool[pos] = key;
         }
@@ -1041,14 +1047,18 @@ size_t fused_smem_bytes(const talon_ctx *c) {
   const size_t tail = sizeof(u64) * EXP_WARPS * (FX_MAX_SPLITS * k + FX_SURV + k) + rows * k * (8 + 8 + 1) +
                       rows * (8 * W + 4 + 4) + 16;
   const size_t ring = sizeof(float) * EXP_WARPS * XS_RING * XS_WTILE;       // the two phases share the space
-  return tail > ring ? tail : ring;
+  return ((tail > ring ? tail : ring) + 15) & ~(size_t)15;
 }
+
+// batches above 32 sequences keep the frontier bases in dynamic shared memory behind that
+size_t fused_base_bytes(int B) { return B > 32 ? sizeof(int) * (MAX_BATCH + 1) : 0; }
 
 }  // namespace
 
 talon_status expand_fused_setup(talon_ctx *c) {
   const size_t bytes = fused_smem_bytes(c);
-  if (cudaFuncSetAttribute(expand_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) !=
+  if (cudaFuncSetAttribute(expand_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(bytes + fused_base_bytes(c->p.batch_max))) !=
       cudaSuccess)
     return TALON_ERR_CUDA;
   int per_sm = 0;
@@ -1077,7 +1087,8 @@ talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float 
   a.row_count = c->d_row_count; a.seq_count = c->d_seq_count; a.status = c->d_status;
   {
     LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
-    launch_kernel(c, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c), st, a);
+    a.base_offset = (int)fused_smem_bytes(c);
+    launch_kernel(c, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c) + fused_base_bytes(c->B), st, a);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;
