@@ -507,12 +507,16 @@ def measure(cfg, args, info, dev, dev_index, peaks, headline: bool, sampler=None
         "value": value, "ms_per_step": seconds / K * 1e3, "steps": K, "repeats": len(reps),
         "spread": (max(reps) - min(reps)) / seconds if len(reps) > 1 else 0.0,
         "warmup": warm, "warmup_requested": args.warmup, "gpu_launches": int(gpu_launches),
-        "sequence_steps_per_s": value * B, "tree_shapes": shapes,
+        "sequence_steps_per_s": value * B, "tree_shapes": shapes, "algorithmic_per_step": work,
         "l2": f"inputs larger than L2: steps rotate over {n_sets} input sets of {per_set / 1e6:.1f} MB "
               f"({n_sets * per_set / 1e6:.0f} MB vs 126 MB L2)",
         "input_sets": n_sets, "timed_wall": (wall0, wall1),
     }
 
+    if args.no_kernel_pass:
+        t.close()
+        res.update({"kernels": {}, "kernels_sum_over_step": None, "kernel_timing": "skipped", "roofline": None})
+        return res
     # ---- each kernel family alone ----
     ms, launches, replays = kernel_pass(t, cfg, sets, main_stream)
     exp_ms = max(ms["reset+expand"] - ms["reset"], 1e-6)
@@ -697,7 +701,10 @@ def run_talon(args):
     subs = [] if (args.config or args.no_sub_configs or info.world > 1) else SUB_CONFIGS
 
     sampler = ClockSampler(dev_index) if info.is_main else None
-    head = measure(synth.CONFIGS[head_name], args, info, dev, dev_index, peaks, True)
+    head_cfg = synth.CONFIGS[head_name]
+    if args.batch is not None:
+        head_cfg = head_cfg.scaled(batch=args.batch)
+    head = measure(head_cfg, args, info, dev, dev_index, peaks, True)
     wall0, wall1 = head.pop("timed_wall")
     clocks = sampler.summary(wall0, wall1) if sampler is not None else None
     others = {}
@@ -707,13 +714,13 @@ def run_talon(args):
         r.pop("timed_wall")
         others[name] = {"workload": workload_text(synth.CONFIGS[name]),
                         **{k: r[k] for k in ("value", "ms_per_step", "steps", "repeats", "spread", "roofline", "kernels",
-                                             "kernels_sum_over_step", "tree_shapes", "input_sets", "gpu_launches")},
+                                             "kernels_sum_over_step", "tree_shapes", "input_sets", "gpu_launches", "algorithmic_per_step")},
                         **({"generation_loop": r["generation_loop"]} if "generation_loop" in r else {})}
     if sampler is not None:
         sampler.stop()
 
     if info.is_main:
-        cfg = synth.CONFIGS[head_name]
+        cfg = head_cfg
         line = {
             "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": info.world, "steps": head["steps"],
             "warmup": head["warmup"], "warmup_requested": head["warmup_requested"], "ms_per_step": head["ms_per_step"],
@@ -728,6 +735,7 @@ def run_talon(args):
             "graph_replay": head.get("graph_replay"), "kernels": head["kernels"], "kernel_timing": head["kernel_timing"],
             "kernels_sum_over_step": head["kernels_sum_over_step"], "sampling_verify": head.get("sampling_verify"),
             "tree_shapes": head["tree_shapes"], "sequence_steps_per_s": head["sequence_steps_per_s"],
+            "algorithmic_per_step": head["algorithmic_per_step"],
             "generation_loop": head.get("generation_loop"),
             "configs": others,
         }
@@ -819,6 +827,10 @@ def main(argv=None):
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-repeat", action="store_true", help="time the K steps once, however short")
     ap.add_argument("--no-loop", action="store_true", help="skip the multi-step generation-loop extra")
+    ap.add_argument("--no-kernel-pass", action="store_true",
+                    help="skip the per-kernel timing pass (for profiler captures of the timed steps alone)")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the workload's batch size (smaller captures of the same kernel shapes)")
     ap.add_argument("--zipf-micro", action="store_true",
                     help="instead of the step benchmark: single-layer expansion latency on Zipf rows")
     args = ap.parse_args(argv)

@@ -847,7 +847,7 @@ expand_fused_kernel(FusedArgs a) {
         unpack_f32x2(add_f32x2(acc0, acc1), s0, s1);
         w.s_t += s0 + s1;
       }
-      refreshed = t < 4 || (t & 3) == 3;         // the threshold is cheap to refresh and pays early
+      refreshed = (t & (t + 1)) == 0 || t == 2;  // after tiles 1, 2, 3, 4, 8, 16, ... of the slice
       // (the first tile has nothing but its own lane maxima to go by: their exact ke-th largest)
       if (refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp, t == 0);
       if (__ballot_sync(FULL, bm >= w.thr_f) != 0u) {
@@ -859,12 +859,13 @@ expand_fused_kernel(FusedArgs a) {
       // tile XS_RING ahead.
       if (lane == 0 && t + XS_RING < nt) issue(t + XS_RING, wt - 1 + XS_RING);
     }
-    if (nt > 0 && !refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp, false);
+    if (nt > 4 && !refreshed) refresh_threshold(w, ke, share_pos, gated, ln_mu, s_wtop, s_wmax, lane, warp, false);
 
     // ---- the warp's survivors -> the CTA pool; its normaliser -> shared memory ----
     {
-      // a warp that could not build a threshold (a short slice) brings its ke best keys only
-      if (w.cnt > 2 * ke + 8) cut_back(buf, ke, w, lane);
+      // a warp that could not build a threshold (a short slice) brings its ke best keys only, so
+      // that eight warps never overflow the pool
+      if (w.cnt > XS_POOL / EXP_WARPS) cut_back(buf, ke, w, lane);
       const int n = w.cnt;
       for (int i = lane; i < n; i += 32) {
         const u64 key = buf[i];
