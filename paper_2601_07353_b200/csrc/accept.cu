@@ -6,6 +6,9 @@
 //                          64-bit atomicMax on a packed (logit, lowest-token-first) key.
 //   accept_walk_kernel   : decodes the keys, then walks from the root along the child whose
 //                          token equals the target's choice until none does.
+// When every CTA of the argmax kernel has one chunk at most (small batches, where a launch costs
+// as much as the work), the CTA that brings a sequence's last chunk does that sequence's walk
+// itself and the second kernel is not launched.
 #include <math_constants.h>
 
 #include "talon_internal.cuh"
@@ -24,9 +27,54 @@ struct ArgmaxArgs {
   int *status;
 };
 
+struct WalkArgs {
+  talon_tree t;
+  int lo_stride;
+  int B, N, max_depth;
+  unsigned long long *best;
+  int32_t *target_tok;      // [B*N] workspace or caller buffer
+  int32_t *accept_len, *accept_nodes, *bonus_tok;
+};
+
+// One warp decodes the keys of sequence b and walks its tree.
+__device__ __forceinline__ void accept_walk(const WalkArgs &a, int b, int lane) {
+  const size_t nb = (size_t)b * a.N;
+  const int n = a.t.n_nodes[b];
+  for (int i = lane; i < a.N; i += 32) {
+    const unsigned long long k = __ldcg(&a.best[nb + i]);
+    a.best[nb + i] = 0ull;                                  // leave the workspace clean
+    a.target_tok[nb + i] = (i < n && k != 0ull) ? (int32_t)key_tok(k) : -1;
+  }
+  __syncwarp();
+  int cur = 0, len = 0;
+  if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1)] = 0;
+  for (int d = 0; d < a.max_depth; ++d) {
+    const int want = a.target_tok[nb + cur];
+    const int lo = a.t.layer_off[b * a.lo_stride + d + 1];
+    const int hi = a.t.layer_off[b * a.lo_stride + d + 2];
+    int found = -1;
+    for (int c0 = lo; c0 < hi; c0 += 32) {
+      const int c = c0 + lane;
+      const bool hit = c < hi && a.t.parent[nb + c] == cur && a.t.token[nb + c] == want;
+      const unsigned m = __ballot_sync(FULL, hit);
+      if (m) { found = c0 + __ffs(m) - 1; break; }
+    }
+    if (found < 0) break;
+    cur = found;
+    ++len;
+    if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1) + len] = cur;
+  }
+  for (int i = len + 1 + lane; i <= a.max_depth; i += 32) a.accept_nodes[(size_t)b * (a.max_depth + 1) + i] = -1;
+  if (lane == 0) {
+    a.accept_len[b] = len;
+    a.bonus_tok[b] = a.target_tok[nb + cur];
+  }
+}
+
 __global__ void __launch_bounds__(EXP_THREADS)
-target_argmax_kernel(ArgmaxArgs a) {
+target_argmax_kernel(ArgmaxArgs a, WalkArgs wa, unsigned int *seq_done, int fold) {
   __shared__ unsigned long long s_key[EXP_WARPS];
+  __shared__ int s_walk;
   pdl_enter();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_items = a.B * a.N * a.splits;
@@ -103,18 +151,21 @@ target_argmax_kernel(ArgmaxArgs a) {
       for (int w = 1; w < EXP_WARPS; ++w) k = s_key[w] > k ? s_key[w] : k;
       if (a.splits == 1) a.best[row] = k;
       else atomicMax(&a.best[row], k);
+      if (fold) {
+        // count the chunk in; whoever brings the sequence's last one walks its tree
+        __threadfence();
+        const unsigned target = (unsigned)(a.n_nodes[b] * a.splits);
+        const unsigned prev = atomicAdd(&seq_done[b], 1u);
+        s_walk = (prev + 1u == target) ? b : -1;
+        if (prev + 1u == target) { seq_done[b] = 0u; __threadfence(); }
+      }
+    }
+    if (fold) {
+      __syncthreads();
+      if (s_walk >= 0 && warp == 0) accept_walk(wa, s_walk, lane);
     }
   }
 }
-
-struct WalkArgs {
-  talon_tree t;
-  int lo_stride;
-  int B, N, max_depth;
-  unsigned long long *best;
-  int32_t *target_tok;      // [B*N] workspace or caller buffer
-  int32_t *accept_len, *accept_nodes, *bonus_tok;
-};
 
 // one warp per sequence
 __global__ void accept_walk_kernel(WalkArgs a) {
@@ -122,38 +173,9 @@ __global__ void accept_walk_kernel(WalkArgs a) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (b >= a.B) return;
-  const size_t nb = (size_t)b * a.N;
-  const int n = a.t.n_nodes[b];
-  for (int i = lane; i < a.N; i += 32) {
-    const unsigned long long k = a.best[nb + i];
-    a.best[nb + i] = 0ull;                                  // leave the workspace clean
-    a.target_tok[nb + i] = (i < n && k != 0ull) ? (int32_t)key_tok(k) : -1;
-  }
-  __syncwarp();
-  int cur = 0, len = 0;
-  if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1)] = 0;
-  for (int d = 0; d < a.max_depth; ++d) {
-    const int want = a.target_tok[nb + cur];
-    const int lo = a.t.layer_off[b * a.lo_stride + d + 1];
-    const int hi = a.t.layer_off[b * a.lo_stride + d + 2];
-    int found = -1;
-    for (int c0 = lo; c0 < hi; c0 += 32) {
-      const int c = c0 + lane;
-      const bool hit = c < hi && a.t.parent[nb + c] == cur && a.t.token[nb + c] == want;
-      const unsigned m = __ballot_sync(FULL, hit);
-      if (m) { found = c0 + __ffs(m) - 1; break; }
-    }
-    if (found < 0) break;
-    cur = found;
-    ++len;
-    if (lane == 0) a.accept_nodes[(size_t)b * (a.max_depth + 1) + len] = cur;
-  }
-  for (int i = len + 1 + lane; i <= a.max_depth; i += 32) a.accept_nodes[(size_t)b * (a.max_depth + 1) + i] = -1;
-  if (lane == 0) {
-    a.accept_len[b] = len;
-    a.bonus_tok[b] = a.target_tok[nb + cur];
-  }
+  accept_walk(a, b, lane);
 }
+
 
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
                            int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
@@ -165,27 +187,29 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   aa.B = c->B; aa.N = c->p.budget; aa.V = c->p.vocab;
   aa.splits = g.splits; aa.chunk_len = g.chunk_len;
   aa.best = c->d_argmax; aa.status = c->d_status;
-  long long items = (long long)rows * g.splits;
-  int grid = c->exp_grid;
-  if (items < grid) grid = (int)items;
-  {
-    LaunchTimer lt(c, TALON_K_ARGMAX, st);
-    launch_kernel(c, target_argmax_kernel, dim3(grid), dim3(EXP_THREADS), 0, st, aa);
-  }
-  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
-
   WalkArgs wa;
   wa.t = *t; wa.lo_stride = c->p.max_depth + 2;
   wa.B = c->B; wa.N = c->p.budget; wa.max_depth = c->p.max_depth;
   wa.best = c->d_argmax; wa.target_tok = target_tok ? target_tok : c->d_target_tok;
   wa.accept_len = accept_len; wa.accept_nodes = accept_nodes; wa.bonus_tok = bonus_tok;
+  long long items = (long long)rows * g.splits;
+  int grid = c->exp_grid;
+  if (items < grid) grid = (int)items;
+  const int fold = items <= grid ? 1 : 0;       // one chunk per CTA at most: the last chunk's CTA walks
+  {
+    LaunchTimer lt(c, TALON_K_ARGMAX, st);
+    launch_kernel(c, target_argmax_kernel, dim3(grid), dim3(EXP_THREADS), 0, st, aa, wa, c->d_walk_count, fold);
+  }
+  if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
+  c->launches += 1;
+  if (fold) return TALON_OK;
   const int warps_per_block = 4;
   {
     LaunchTimer lt(c, TALON_K_WALK, st);
     launch_kernel(c, accept_walk_kernel, dim3((c->B + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, st, wa);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
-  c->launches += 2;
+  c->launches += 1;
   return TALON_OK;
 }
 

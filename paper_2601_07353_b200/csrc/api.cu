@@ -145,6 +145,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
   alloc((void **)&c->d_seq_count, sizeof(unsigned int) * (size_t)p->batch_max);
   alloc((void **)&c->d_argmax, sizeof(unsigned long long) * nrow);
   alloc((void **)&c->d_target_tok, sizeof(int32_t) * nrow);
+  alloc((void **)&c->d_walk_count, sizeof(unsigned int) * (size_t)p->batch_max);
   alloc((void **)&c->d_samp_ms, sizeof(float2) * nrow * talon::EXP_MAX_SPLITS);
   c->attn_o_elems = talon::attention_workspace_elems(c, &c->attn_ml_elems);
   alloc((void **)&c->d_attn_o, sizeof(float) * c->attn_o_elems);
@@ -154,6 +155,7 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
          cudaMemset(c->d_row_count, 0, sizeof(unsigned int) * (size_t)c->rows_cap) == cudaSuccess &&
          cudaMemset(c->d_argmax, 0, sizeof(unsigned long long) * nrow) == cudaSuccess &&
          cudaMemset(c->d_seq_count, 0, sizeof(unsigned int) * (size_t)p->batch_max) == cudaSuccess &&
+         cudaMemset(c->d_walk_count, 0, sizeof(unsigned int) * (size_t)p->batch_max) == cudaSuccess &&
          cudaMemset(c->d_part_keys, 0, sizeof(unsigned long long) * (size_t)c->items_cap * c->key_stride) == cudaSuccess &&
          talon::expand_setup(c) == TALON_OK && talon::attention_mma_setup() == TALON_OK &&
          talon::attention_tc_setup() == TALON_OK &&
@@ -173,7 +175,7 @@ talon_status talon_destroy(talon_ctx *c) {
   cudaSetDevice(c->device);
   cudaFree(c->d_status); cudaFree(c->d_prefix_len); cudaFree(c->d_part_keys); cudaFree(c->d_part_ms);
   cudaFree(c->d_row_keys); cudaFree(c->d_row_lse); cudaFree(c->d_row_score); cudaFree(c->d_row_count); cudaFree(c->d_seq_count); cudaFree(c->d_argmax);
-  cudaFree(c->d_target_tok); cudaFree(c->d_samp_ms); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
+  cudaFree(c->d_target_tok); cudaFree(c->d_walk_count); cudaFree(c->d_samp_ms); cudaFree(c->d_attn_o); cudaFree(c->d_attn_ml);
   free_stage(c->stage);
   talon_timing_enable(c, 0, 0u);
   if (c->graphs) {

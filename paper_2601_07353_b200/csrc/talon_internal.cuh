@@ -127,6 +127,7 @@ struct talon_ctx {
   // verification workspace
   unsigned long long *d_argmax;      // [batch_max * N] packed (logit, token) maxima
   int32_t *d_target_tok;             // [batch_max * N]
+  unsigned int *d_walk_count;        // [batch_max] argmax chunks finished per sequence (zero between calls)
   float2 *d_samp_ms;                 // [batch_max * N, EXP_MAX_SPLITS] per-chunk (max, sum) of target rows
   float *d_attn_o;                   // split-KV partial outputs
   float2 *d_attn_ml;                 // split-KV partial (max, sum)
