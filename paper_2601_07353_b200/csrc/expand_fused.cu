@@ -260,6 +260,7 @@ __device__ inline double f64_unord(u64 o) {
 struct SpanGeom {
   unsigned span;       // elements of the line per CTA
   unsigned pitch;      // elements of the line per row (>= the row length)
+  unsigned per_row;    // chunks per row when no span crosses a row, else 0
 };
 
 __device__ inline unsigned div_u64(unsigned long long a, unsigned b) {
@@ -274,18 +275,25 @@ __device__ inline SpanGeom span_geom(int total_rows, int vocab, int grid, int ma
     const unsigned S = max(1u, min(min(per_row, (unsigned)max_split), vp / 4096u));
     g.span = ((vp + S - 1u) / S + 3u) & ~3u;
     g.pitch = S * g.span;
+    g.per_row = S;
   } else {
     const unsigned long long line = (unsigned long long)total_rows * vp;
     const unsigned span = (div_u64(line + grid - 1, (unsigned)grid) + 3u) & ~3u;
     const unsigned span_min = max(4096u, ((vp + FX_MAX_SPLITS - 2) / (FX_MAX_SPLITS - 1) + 3u) & ~3u);
     g.span = max(span, span_min);
     g.pitch = vp;
+    g.per_row = 0u;
   }
   return g;
 }
 
 // First chunk-result index and number of chunks of packed row `row`.
 __device__ inline void row_chunks(const SpanGeom &g, int row, int &item0, int &S) {
+  if (g.per_row) {                       // equal chunks of whole rows: no division
+    item0 = row * (int)g.per_row + row;
+    S = (int)g.per_row;
+    return;
+  }
   const unsigned long long lo = (unsigned long long)row * g.pitch;
   const unsigned first = div_u64(lo, g.span), last = div_u64(lo + g.pitch - 1, g.span);
   item0 = (int)first + row;
@@ -515,14 +523,17 @@ __device__ __forceinline__ bool merge_row(const FusedArgs &a, size_t item0, int 
       }
     }
   }
-  float mx = ms.x;
+  static_assert(FX_MAX_SPLITS <= 16, "the chunk statistics are reduced over 16 lanes");
+  float mx = ms.x;                                                      // lanes >= S hold -inf and 0
 #pragma unroll
-  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+  for (int o = 8; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+  mx = __shfl_sync(FULL, mx, 0);
   double t = 0.0;
   if (ms.y != ms.y) t = (double)ms.y;                                   // NaN or +inf logit in the chunk
   else if (ms.x > -CUDART_INF_F) t = (double)ms.y * (double)exp2f((ms.x - mx) * LOG2E_F);
 #pragma unroll
-  for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
+  for (int o = 8; o; o >>= 1) t += __shfl_xor_sync(FULL, t, o);
+  t = __shfl_sync(FULL, t, 0);
   const bool finite = (t > 0.0) && (t < CUDART_INF) && (mx < CUDART_INF_F) && (mx > -CUDART_INF_F);
 
   if (S > 1) {
