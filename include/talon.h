@@ -178,6 +178,16 @@ talon_status talon_accept(talon_ctx *ctx, const talon_tree *tree, const float *t
                           int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                           int32_t *accept_nodes, int32_t *bonus_tok, void *stream);
 
+/* talon_build_tree (without the dense mask) and talon_accept in one call, for the tail of a step:
+ * the warp that walks a sequence's tree first writes that sequence's positions, sentinel slots and
+ * closed layer offsets, so the closing kernel is not launched.  Nothing between the last expansion
+ * layer and this call may need what talon_build_tree writes (talon_tree_attention does not: it
+ * reads sizes and mask rows).  Arguments, results and errors as talon_accept; talon_step and
+ * talon_loop end their steps with it. */
+talon_status talon_close_and_accept(talon_ctx *ctx, const talon_tree *tree, const float *target_logits,
+                                    int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
+                                    int32_t *accept_nodes, int32_t *bonus_tok, void *stream);
+
 /* Sampling verification (Appendix B steps 1-3, the paper's temperature-1 setting; the appendix
  * names the steps and the property -- what is emitted is distributed exactly as the target
  * model's own samples -- and leaves the procedure to the literature it cites).  With p the

@@ -8,7 +8,9 @@
 //                          token equals the target's choice until none does.
 // When every CTA of the argmax kernel has one chunk at most (small batches, where a launch costs
 // as much as the work), the CTA that brings a sequence's last chunk does that sequence's walk
-// itself and the second kernel is not launched.
+// itself and the second kernel is not launched.  Inside a whole step the walk's warp also closes
+// the tree (positions, sentinel slots, the unused tail of the layer offsets), which saves the
+// launch of the closing kernel: nothing between the last expansion layer and the walk reads those.
 #include <math_constants.h>
 
 #include "talon_internal.cuh"
@@ -34,12 +36,40 @@ struct WalkArgs {
   unsigned long long *best;
   int32_t *target_tok;      // [B*N] workspace or caller buffer
   int32_t *accept_len, *accept_nodes, *bonus_tok;
+  // closing pass folded into the walk (close_tree != 0)
+  int close_tree, W, layers_run;
+  const int32_t *prefix_len;
 };
+
+// The closing pass over the node slots of sequence b (what build_tree_kernel writes there):
+// positions of the tree's nodes, sentinels in the unused slots.  The walk reads none of it.
+__device__ __forceinline__ void close_slots(const WalkArgs &a, int b, int first, int step) {
+  const size_t nb = (size_t)b * a.N;
+  const int n = a.t.n_nodes[b];
+  const int L = a.prefix_len[b];
+  for (int i = first; i < a.N; i += step) {
+    if (i < n) {
+      a.t.position[nb + i] = L + a.t.depth[nb + i];
+    } else {
+      a.t.token[nb + i] = -1;
+      a.t.parent[nb + i] = -1;
+      a.t.depth[nb + i] = -1;
+      a.t.position[nb + i] = -1;
+      a.t.score[nb + i] = -CUDART_INF;
+      for (int w = 0; w < a.W; ++w) a.t.mask[(nb + i) * a.W + w] = ((i >> 6) == w) ? (1ull << (i & 63)) : 0ull;
+    }
+  }
+}
 
 // One warp decodes the keys of sequence b and walks its tree.
 __device__ __forceinline__ void accept_walk(const WalkArgs &a, int b, int lane) {
   const size_t nb = (size_t)b * a.N;
   const int n = a.t.n_nodes[b];
+  if (a.close_tree) {
+    // layers that were never launched: their offsets close at the tree's size (the walk reads them)
+    for (int i = a.layers_run + 2 + lane; i < a.lo_stride; i += 32) a.t.layer_off[b * a.lo_stride + i] = n;
+    __syncwarp();
+  }
   for (int i = lane; i < a.N; i += 32) {
     const unsigned long long k = __ldcg(&a.best[nb + i]);
     a.best[nb + i] = 0ull;                                  // leave the workspace clean
@@ -162,7 +192,10 @@ target_argmax_kernel(ArgmaxArgs a, WalkArgs wa, unsigned int *seq_done, int fold
     }
     if (fold) {
       __syncthreads();
-      if (s_walk >= 0 && warp == 0) accept_walk(wa, s_walk, lane);
+      if (s_walk >= 0) {
+        if (warp == 0) accept_walk(wa, s_walk, lane);
+        else if (wa.close_tree) close_slots(wa, s_walk, tid - 32, EXP_THREADS - 32);   // beside the walk
+      }
     }
   }
 }
@@ -173,13 +206,45 @@ __global__ void accept_walk_kernel(WalkArgs a) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (b >= a.B) return;
+  // the closing pass needs each node's depth: the loads are issued before the walk (a chain of
+  // dependent L2 trips) and their results are used after it
+  constexpr int PER = (MAX_BUDGET + 31) / 32;
+  int dep[PER];
+  int L = 0, n = 0;
+  if (a.close_tree) {
+    n = a.t.n_nodes[b];
+    L = a.prefix_len[b];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int i = lane + 32 * k;
+      dep[k] = (i < n) ? a.t.depth[(size_t)b * a.N + i] : -1;
+    }
+  }
   accept_walk(a, b, lane);
+  if (a.close_tree) {
+    const size_t nb = (size_t)b * a.N;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int i = lane + 32 * k;
+      if (i >= a.N) continue;
+      if (i < n) {
+        a.t.position[nb + i] = L + dep[k];
+      } else {
+        a.t.token[nb + i] = -1;
+        a.t.parent[nb + i] = -1;
+        a.t.depth[nb + i] = -1;
+        a.t.position[nb + i] = -1;
+        a.t.score[nb + i] = -CUDART_INF;
+        for (int w = 0; w < a.W; ++w) a.t.mask[(nb + i) * a.W + w] = ((i >> 6) == w) ? (1ull << (i & 63)) : 0ull;
+      }
+    }
+  }
 }
 
 
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
                            int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
-                           int32_t *bonus_tok, cudaStream_t st) {
+                           int32_t *bonus_tok, cudaStream_t st, bool close_tree) {
   const int rows = c->B * c->p.budget;
   const LayerGeom g = make_geom(rows, c->p.vocab, c->exp_grid);
   ArgmaxArgs aa;
@@ -192,6 +257,7 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
   wa.B = c->B; wa.N = c->p.budget; wa.max_depth = c->p.max_depth;
   wa.best = c->d_argmax; wa.target_tok = target_tok ? target_tok : c->d_target_tok;
   wa.accept_len = accept_len; wa.accept_nodes = accept_nodes; wa.bonus_tok = bonus_tok;
+  wa.close_tree = close_tree ? 1 : 0; wa.W = c->W; wa.layers_run = c->layers_run; wa.prefix_len = c->d_prefix_len;
   long long items = (long long)rows * g.splits;
   int grid = c->exp_grid;
   if (items < grid) grid = (int)items;

@@ -262,15 +262,28 @@ talon_status talon_tree_attention_paged(talon_ctx *c, const talon_tree *t, const
                                  kv_stride_h, max_prefix_len, sm_scale, out, (cudaStream_t)stream);
 }
 
-talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
-                          int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
-                          void *stream) {
+// close_tree: the walk also does talon_build_tree's writes (used inside a whole step)
+static talon_status accept_checked(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                                   int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
+                                   int32_t *bonus_tok, void *stream, bool close_tree) {
   if (!c || !tree_complete(t) || !target_logits || !accept_len || !accept_nodes || !bonus_tok)
     return TALON_ERR_INVALID_ARG;
   if (c->B < 1) return TALON_ERR_INVALID_ARG;
   if (row_stride < c->p.vocab || (row_stride & 3) || !aligned16(target_logits)) return TALON_ERR_INVALID_ARG;
   return talon::launch_accept(c, t, target_logits, row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
-                              (cudaStream_t)stream);
+                              (cudaStream_t)stream, close_tree);
+}
+
+talon_status talon_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                          int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes, int32_t *bonus_tok,
+                          void *stream) {
+  return accept_checked(c, t, target_logits, row_stride, target_tok, accept_len, accept_nodes, bonus_tok, stream, false);
+}
+
+talon_status talon_close_and_accept(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
+                                    int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
+                                    int32_t *bonus_tok, void *stream) {
+  return accept_checked(c, t, target_logits, row_stride, target_tok, accept_len, accept_nodes, bonus_tok, stream, true);
 }
 
 talon_status talon_accept_sample(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
@@ -458,13 +471,14 @@ static talon_status step_enqueue(talon_ctx *c, const talon_tree *t, int32_t B, c
   talon_status r = talon_reset(c, t, root_tok, prefix_len, B, stream);
   for (int d = 0; r == TALON_OK && d < n_layers; ++d)
     r = talon_expand_layer(c, t, draft_logits, draft_row_stride, c->p.budget, TALON_ROWS_BY_NODE, stream);
-  if (r == TALON_OK) r = talon_build_tree(c, t, nullptr, stream);
+  // (no separate closing launch: the attention needs only sizes and mask rows, and the accept walk
+  // writes positions and sentinel slots before it walks)
   if (r == TALON_OK)
     r = talon_tree_attention(c, t, q, k_prefix, v_prefix, k_tree, v_tree, kv_start, kv_tokens, kv_stride_t, kv_stride_h,
                              max_prefix_len, sm_scale, out, stream);
   if (r == TALON_OK)
-    r = talon_accept(c, t, target_logits, target_row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
-                     stream);
+    r = accept_checked(c, t, target_logits, target_row_stride, target_tok, accept_len, accept_nodes, bonus_tok,
+                       stream, true);
   return r;
 }
 

@@ -215,7 +215,7 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
                                  int splits, int m_blocks, cudaStream_t st);
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
-                           int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st);
+                           int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st, bool close_tree = false);
 talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float *target_logits, int64_t row_stride,
                                   double temperature, const double *u_accept, const double *u_sample,
                                   int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, cudaStream_t st);

@@ -53,6 +53,7 @@ _lib.talon_loop.argtypes = ([_vp, _TP, _i32, _i32, _vp, _vp, _vp, _i64, _i64, _i
 _lib.talon_loop_metrics.argtypes = [_vp, _i32, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
 _lib.talon_tree_attention.argtypes = [_vp, _TP, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _f32, _vp, _vp]
 _lib.talon_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.talon_close_and_accept.argtypes = [_vp, _TP, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_accept_sample.argtypes = [_vp, _TP, _vp, _i64, C.c_double, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.talon_commit.argtypes = [_vp, _TP] + [_vp] * 9 + [_i64, _i64, _i64, _vp, _vp, _vp, _vp]
 _lib.talon_poll_status.argtypes = [_vp, _vp]
@@ -73,7 +74,8 @@ for _n in ("talon_create", "talon_destroy", "talon_reset", "talon_expand_layer",
            "talon_build_tree", "talon_tree_attention", "talon_accept", "talon_poll_status", "talon_step_host",
            "talon_step", "talon_timing_enable", "talon_timing_read", "talon_timing_pause",
            "talon_target_argmax_noalloc", "talon_accept_sample", "talon_commit", "talon_prune_tree",
-           "talon_tree_attention_paged", "talon_commit_paged", "talon_loop", "talon_loop_metrics"):
+           "talon_tree_attention_paged", "talon_commit_paged", "talon_loop", "talon_loop_metrics",
+           "talon_close_and_accept"):
     getattr(_lib, _n).restype = C.c_int
 
 EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer", "talon_layers_run",
@@ -82,7 +84,7 @@ EXPORTED = ["talon_create", "talon_destroy", "talon_reset", "talon_expand_layer"
             "talon_kernel_name",
             "talon_launch_count", "talon_status_string", "talon_target_argmax_noalloc", "talon_accept_sample",
             "talon_commit", "talon_prune_tree", "talon_tree_attention_paged", "talon_commit_paged", "talon_loop",
-            "talon_loop_metrics"]
+            "talon_loop_metrics", "talon_close_and_accept"]
 PAGE_TOKENS = 128
 NOALLOC_MAX_ROWS = 8192
 N_KERNELS = 11
@@ -227,6 +229,15 @@ class Talon:
         _check(_lib.talon_accept(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, _ptr(target_tok),
                                  _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok), _stream(self.device)),
                "talon_accept")
+
+    def close_and_accept(self, tree: Tree, target_logits, accept_len, accept_nodes, bonus_tok, target_tok=None,
+                         row_stride: Optional[int] = None):
+        ts = tree.struct()
+        if row_stride is None:
+            row_stride = target_logits.stride(-2)
+        _check(_lib.talon_close_and_accept(self._ctx, C.byref(ts), _ptr(target_logits), row_stride, _ptr(target_tok),
+                                           _ptr(accept_len), _ptr(accept_nodes), _ptr(bonus_tok), _stream(self.device)),
+               "talon_close_and_accept")
 
     def accept_sample(self, tree: Tree, target_logits, temperature: float, u_accept, u_sample, accept_len,
                       accept_nodes, out_tok, row_stride: Optional[int] = None):

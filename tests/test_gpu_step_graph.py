@@ -119,3 +119,47 @@ def test_more_argument_sets_than_graph_slots():
         assert torch.equal(o, want)
     assert torch.equal(wl.tree.token, want_tok)
     t.close()
+
+
+@pytest.mark.parametrize("batch,layers", [(1, None), (3, 2), (24, None), (24, 1)])
+def test_close_and_accept_equals_build_then_accept(batch, layers):
+    """The tail of a step in one call: the accept walk's warp writes what talon_build_tree writes
+    (positions, sentinel slots, the unused tail of the layer offsets) before it walks.  Small batches
+    take the route where the argmax kernel's last CTA walks, large ones the separate walk kernel;
+    fewer layers than D_max leave layer offsets for the closing pass to fill."""
+    from paper_2601_07353_b200 import talon, workload
+    cfg = synth.CONFIGS["tiny"].scaled(batch=batch, prefix_min=20, prefix_max=300, vocab=8000)
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, GP.SEED)
+    n_layers = cfg.max_depth if layers is None else layers
+    tr = wl.tree
+
+    def head():
+        for x in (tr.token, tr.parent, tr.depth, tr.position, tr.layer_off, tr.mask, wl.accept_len, wl.accept_nodes,
+                  wl.bonus_tok, wl.target_tok):
+            x.fill_(77)                              # stale contents everywhere the tail must write
+        tr.score.fill_(7.0)
+        t.reset(tr, wl.root_tok, wl.prefix_len)
+        for _ in range(n_layers):
+            t.expand_layer(tr, wl.draft)
+
+    head()
+    t.build_tree(tr)
+    t.accept(tr, wl.target, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok)
+    torch.cuda.synchronize()
+    assert t.poll_status() == talon.OK
+    want = _snapshot(wl)
+    head()
+    before = t.launch_count()
+    t.close_and_accept(tr, wl.target, wl.accept_len, wl.accept_nodes, wl.bonus_tok, wl.target_tok)
+    torch.cuda.synchronize()
+    assert t.poll_status() == talon.OK
+    assert t.launch_count() - before in (1, 2)       # argmax (+ walk): no closing launch
+    names = ("n_nodes", "token", "parent", "depth", "position", "layer_off", "score", "mask", "out", "accept_len",
+             "accept_nodes", "bonus_tok", "target_tok")
+    for name, a, b in zip(names, want, _snapshot(wl)):
+        if name == "score":
+            assert torch.equal(a.view(torch.int64), b.view(torch.int64)), name     # -inf sentinels included
+        else:
+            assert torch.equal(a, b), name
+    t.close()
