@@ -545,9 +545,9 @@ __device__ __forceinline__ bool merge_row(const FusedArgs &a, size_t item0, int 
     const u64 head = lane < S ? st[lane] : 0ull;
     u64 tau = lane < S ? st[(ke - 1) * FX_MAX_SPLITS + lane] : 0ull;
     if (S >= ke) {
-      int cnt = 0;
-#pragma unroll 8
-      for (int o = 0; o < 32; ++o) cnt += (shfl_u64(head, o) > head) ? 1 : 0;
+      int cnt = 0;                                 // (lanes past the chunks hold 0 and count for nothing)
+#pragma unroll
+      for (int o = 0; o < FX_MAX_SPLITS; ++o) cnt += (shfl_u64(head, o) > head) ? 1 : 0;
       if (cnt == ke - 1) tau = umax64(tau, head);
     }
     tau = warp_max_u64(tau);
@@ -679,6 +679,7 @@ __device__ void select_and_append(const FusedArgs &a, const TailSmem &sm, int b,
     const int j = c / k;
     const int tok = (int)key_tok(sm.row_keys[c]);
     int r = 0;
+#pragma unroll 4
     for (int i = 0; i < ke; ++i) {
       const int o = j * k + i;
       r += ((sm.state[o] & 4) && (int)key_tok(sm.row_keys[o]) < tok) ? 1 : 0;
