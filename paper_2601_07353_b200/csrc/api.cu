@@ -119,6 +119,9 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     c->expand_max_split = ms ? std::atoi(ms) : talon::FX_MAX_SPLITS - 1;
     if (c->expand_max_split < 1) c->expand_max_split = 1;
     if (c->expand_max_split > talon::FX_MAX_SPLITS - 1) c->expand_max_split = talon::FX_MAX_SPLITS - 1;
+    const char *ao = std::getenv("TALON_ARGMAX_OVERSPLIT");
+    c->argmax_oversplit = ao ? std::atoi(ao) : 4;
+    if (c->argmax_oversplit < 1) c->argmax_oversplit = 1;
     const char *e = std::getenv("TALON_PDL");
     c->pdl = !e ? -1 : (e[0] == '1' ? 1 : 0);
     const char *g = std::getenv("TALON_STEP_GRAPH");

@@ -121,6 +121,7 @@ struct talon_ctx {
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int argmax_oversplit;              // target argmax: chunk rounds per CTA when the rows outnumber the grid
   int expand_max_split;              // fused kernel: chunks a row is cut into at most when the grid has room
   int attn_min_tiles;                // split-KV: key tiles a CTA should at least own
   int pdl;                           // programmatic stream serialization: 1 on, 0 off, -1 on for small batches
