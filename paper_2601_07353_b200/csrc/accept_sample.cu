@@ -438,7 +438,10 @@ talon_status launch_accept_sample(talon_ctx *c, const talon_tree *t, const float
                                   int32_t *accept_len, int32_t *accept_nodes, int32_t *out_tok, cudaStream_t st) {
   if (c->p.vocab > SAMP_MAX_GROUPS * SAMP_GROUP || c->p.budget > SAMP_MAX_NODES) return TALON_ERR_UNSUPPORTED;
   const int rows = c->B * c->p.budget;
-  const LayerGeom g = make_geom(rows, c->p.vocab, c->exp_grid);
+  LayerGeom g = make_geom(rows, c->p.vocab, c->exp_grid);
+  // (as in the greedy arg-max pass: finer chunks when the rows outnumber the grid)
+  if ((long long)rows * g.splits > c->exp_grid && c->argmax_oversplit > 1)
+    g = make_geom(rows, c->p.vocab, c->exp_grid * c->argmax_oversplit);
   StatsArgs sa;
   sa.logits = target_logits; sa.row_stride = row_stride; sa.n_nodes = t->n_nodes;
   sa.B = c->B; sa.N = c->p.budget; sa.V = c->p.vocab;
