@@ -119,6 +119,8 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     c->expand_max_split = ms ? std::atoi(ms) : talon::FX_MAX_SPLITS - 1;
     if (c->expand_max_split < 1) c->expand_max_split = 1;
     if (c->expand_max_split > talon::FX_MAX_SPLITS - 1) c->expand_max_split = talon::FX_MAX_SPLITS - 1;
+    const char *fs = std::getenv("TALON_ATTN_SPLITS");
+    c->attn_force_splits = fs ? std::atoi(fs) : 0;
     const char *ao = std::getenv("TALON_ARGMAX_OVERSPLIT");
     c->argmax_oversplit = ao ? std::atoi(ao) : 4;
     if (c->argmax_oversplit < 1) c->argmax_oversplit = 1;

@@ -383,6 +383,7 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
       };
       if (tiles >= 32 && cost(2) < cost(1)) sp = 2;
     }
+    if (c->attn_force_splits > 0) sp = c->attn_force_splits;
     while (sp > 1 && (size_t)a.m_blocks * c->B * a.Hkv * sp * AT_BM > c->attn_ml_elems) --sp;
     a.splits = sp;
     talon_status r = launch_attention_tc(c, t, q, kp, vp, kt, vt, kv_start, block_table, bt_stride, stride_t, stride_h, kv_tokens,

@@ -121,6 +121,7 @@ struct talon_ctx {
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int attn_force_splits;             // > 0: key ranges per (sequence, head, query tiles), for experiments
   int argmax_oversplit;              // target argmax: chunk rounds per CTA when the rows outnumber the grid
   int expand_max_split;              // fused kernel: chunks a row is cut into at most when the grid has room
   int attn_min_tiles;                // split-KV: key tiles a CTA should at least own
