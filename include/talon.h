@@ -42,7 +42,8 @@ typedef enum {
   TALON_ERR_INVALID_ARG = 1, /* null pointer, size out of range, misaligned row          */
   TALON_ERR_CAPACITY = 2,    /* request exceeds what the context was created for          */
   TALON_ERR_CUDA = 3,        /* a CUDA runtime call failed (see stderr for the message)   */
-  TALON_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up                        */
+  TALON_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up: the tree arrays and   */
+                             /* outputs of that step are undefined, call talon_reset     */
   TALON_ERR_NONFINITE = 5,   /* NaN / +inf logit, or a row holding only -inf              */
   TALON_ERR_UNSUPPORTED = 6  /* valid in the paper, not built (e.g. head_dim != 128)      */
 } talon_status;
