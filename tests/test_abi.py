@@ -35,6 +35,18 @@ def test_status_strings_and_host_side_argument_checks():
     assert lib.talon_expand_layer(None, None, None, ctypes.c_int64(0), 0, 0, None) == 1
     assert lib.talon_build_tree(None, None, None, None) == 1
     assert lib.talon_poll_status(None, None) == 1
+    # the later additions reject a missing context the same way
+    i64 = ctypes.c_int64
+    assert lib.talon_accept(None, None, None, i64(0), None, None, None, None, None) == 1
+    assert lib.talon_close_and_accept(None, None, None, i64(0), None, None, None, None, None) == 1
+    assert lib.talon_prune_tree(None, None, 1, None) == 1
+    assert lib.talon_loop_metrics(None, 1, ctypes.c_double(0.05), None, None, None) == 1
+    # delta, tau and R of Eq. 6-7 are host arithmetic behind the C ABI: 3 verification passes, 12 draft
+    # passes, 9 tokens give delta 4, tau 3 and R = 3 / (1 + 0.1 * 4)
+    cnt = (i64 * 6)(1, 5, 2, 2, 7, 7)
+    d, tau, r = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    assert lib.talon_loop_metrics(cnt, 2, ctypes.c_double(0.1), ctypes.byref(d), ctypes.byref(tau), ctypes.byref(r)) == 0
+    assert d.value == 4.0 and tau.value == 3.0 and abs(r.value - 3.0 / 1.4) < 1e-15
 
 
 def test_binding_names_match_header():
