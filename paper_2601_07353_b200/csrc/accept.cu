@@ -246,7 +246,9 @@ talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *targe
                            int32_t *target_tok, int32_t *accept_len, int32_t *accept_nodes,
                            int32_t *bonus_tok, cudaStream_t st, bool close_tree) {
   const int rows = c->B * c->p.budget;
-  LayerGeom g = make_geom(rows, c->p.vocab, c->exp_grid);
+  // Fewer rows than CTAs: as many chunks per row as keep rows x chunks within the grid (rounded
+  // down), so that every CTA has one chunk and the last chunk's CTA can do the walk.
+  LayerGeom g = make_geom(rows, c->p.vocab, rows <= c->exp_grid ? c->exp_grid - rows + 1 : c->exp_grid);
   // More rows than half the grid: with one chunk per CTA round the last round leaves most SMs
   // idle (960 rows on 592 CTAs are 1.6 rounds); finer chunks keep every CTA streaming to the end.
   if ((long long)rows * g.splits > c->exp_grid && c->argmax_oversplit > 1)
