@@ -53,3 +53,21 @@ def test_binding_names_match_header():
     src = open(os.path.join(ROOT, "paper_2601_07353_b200", "talon.py")).read()
     for n in declared_functions():
         assert n in src, f"binding does not mention {n}"
+
+
+def test_the_product_has_no_cpu_route():
+    """The package never imports the oracle, and without a CUDA device a context cannot be made."""
+    import glob
+    import pytest
+    import torch
+    for path in glob.glob(os.path.join(ROOT, "paper_2601_07353_b200", "*.py")):
+        src = open(path).read()
+        assert "oracle" not in src or "talon_oracle" not in src, f"{path} mentions the oracle module"
+        assert not re.search(r"^\s*(from|import)\s+oracle\b", src, flags=re.M), f"{path} imports the oracle"
+    for path in glob.glob(os.path.join(ROOT, "oracle", "*.py")):
+        src = open(path).read()
+        assert not re.search(r"^\s*(from|import)\s+paper_2601_07353_b200\b", src, flags=re.M), f"{path} imports the package"
+    if not torch.cuda.is_available():
+        from paper_2601_07353_b200 import talon
+        with pytest.raises(RuntimeError):
+            talon.Talon(batch_max=1, vocab=100, budget=8, root_topk=4, cand_topk=4, max_depth=4, n_q_heads=4, n_kv_heads=2)
