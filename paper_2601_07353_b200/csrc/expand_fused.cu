@@ -1101,7 +1101,7 @@ talon_status launch_expand_fused(talon_ctx *c, const talon_tree *t, const float 
   {
     LaunchTimer lt(c, TALON_K_EXPAND_ROWS, st);
     a.base_offset = (int)fused_smem_bytes(c);
-    launch_kernel(c, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c) + fused_base_bytes(c->B), st, a);
+    launch_kernel_pdl(c, true, expand_fused_kernel, dim3(grid), dim3(EXP_THREADS), fused_smem_bytes(c) + fused_base_bytes(c->B), st, a);
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;

@@ -164,9 +164,12 @@ __device__ __forceinline__ void pdl_enter() {
 // overlapped launch latency is a gain, while at larger batches the early-scheduled CTAs of the next
 // kernel take SM slots from the running one.
 constexpr int PDL_AUTO_BATCH = 4;
+// `chain` marks the launches of a chain of short dependent kernels (the expansion layers): there
+// the overlap of launch latency pays at every batch size (a layer that finds every tree full costs
+// little more than its launch), while behind the long verification kernels it does not.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                 cudaStream_t st, Args &&...args) {
+inline cudaError_t launch_kernel_pdl(const talon_ctx *c, bool chain, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                     size_t smem, cudaStream_t st, Args &&...args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -176,8 +179,13 @@ inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), d
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (c->pdl == 1 || (c->pdl < 0 && c->B <= PDL_AUTO_BATCH)) ? 1 : 0;
+  cfg.numAttrs = (c->pdl == 1 || (c->pdl < 0 && (c->B <= PDL_AUTO_BATCH || chain))) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(const talon_ctx *c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, Args &&...args) {
+  return launch_kernel_pdl(c, false, kernel, grid, block, smem, st, static_cast<Args &&>(args)...);
 }
 
 // Brackets one kernel launch with a pair of CUDA events on the launching stream when timing
