@@ -119,6 +119,13 @@ talon_status talon_create(talon_ctx **out_ctx, const talon_params *p, int device
     c->expand_max_split = ms ? std::atoi(ms) : talon::FX_MAX_SPLITS - 1;
     if (c->expand_max_split < 1) c->expand_max_split = 1;
     if (c->expand_max_split > talon::FX_MAX_SPLITS - 1) c->expand_max_split = talon::FX_MAX_SPLITS - 1;
+    const char *ac = std::getenv("TALON_ATTN_CLUSTER");
+    c->attn_cluster = ac ? std::atoi(ac) : 1;
+    for (int i = 0; i < 9; ++i) c->attn_cluster_ok[i] = -1;
+    const char *cc = std::getenv("TALON_ATTN_CLUSTER_CAP");
+    c->attn_cluster_cap = cc ? std::atoi(cc) : 32;
+    const char *cr = std::getenv("TALON_ATTN_CLUSTER_MIN_ROWS");
+    c->attn_cluster_min_rows = cr ? std::atoll(cr) : 8192;
     const char *fs = std::getenv("TALON_ATTN_SPLITS");
     c->attn_force_splits = fs ? std::atoi(fs) : 0;
     const char *ao = std::getenv("TALON_ARGMAX_OVERSPLIT");

@@ -370,6 +370,11 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
       const int by_tiles = (tiles + c->attn_min_tiles - 1) / c->attn_min_tiles;
       if (sp > by_tiles) sp = by_tiles;
       if (sp < 1) sp = 1;
+      // up to eight key ranges can merge inside one thread-block cluster, which saves the merge
+      // kernel; a ninth range is worth less than that
+      if (c->attn_cluster && sp > 8 && sp <= c->attn_cluster_cap &&
+          (c->attn_cluster == 2 || (long long)c->B * a.Hkv * a.g * a.N * 8 >= c->attn_cluster_min_rows))
+        sp = 8;
     } else if (ctas % c->sm_count) {
       // More CTAs than SMs and a ragged last wave: halving the key ranges can fill it (512 CTAs on
       // 148 SMs are 4 waves of 257 tiles, 1024 half CTAs are 7 waves of 129).  Cost model in key
@@ -386,10 +391,11 @@ talon_status launch_attention(talon_ctx *c, const talon_tree *t, const void *q, 
     if (c->attn_force_splits > 0) sp = c->attn_force_splits;
     while (sp > 1 && (size_t)a.m_blocks * c->B * a.Hkv * sp * AT_BM > c->attn_ml_elems) --sp;
     a.splits = sp;
+    int merged = 0;
     talon_status r = launch_attention_tc(c, t, q, kp, vp, kt, vt, kv_start, block_table, bt_stride, stride_t, stride_h, kv_tokens,
-                                         max_prefix_len, sm_scale, out, sp, a.m_blocks, st);
+                                         max_prefix_len, sm_scale, out, sp, a.m_blocks, st, &merged);
     if (r != TALON_OK) return r;
-    if (sp > 1) {
+    if (sp > 1 && !merged) {
       const int64_t rows = (int64_t)c->B * a.Hkv * a.g * a.N;
       const int wpb = 8;
       LaunchTimer lt(c, TALON_K_COMBINE, st);

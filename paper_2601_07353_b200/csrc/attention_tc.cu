@@ -46,6 +46,9 @@ constexpr int TC_SMEM = (2 + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 + TC_NBARS * 
 constexpr uint32_t TC_TMEM_COLS = 512;     // O0 | O1 | S0 | S1, 128 fp32 columns each
 constexpr float TC_RESCALE_GAP = 8.f;      // raise the reference maximum only beyond 2^8
 constexpr long long TC_WAIT_CYCLES = 4000000000ll;   // ~2 s: far beyond any legitimate wait
+constexpr int TC_XO_PITCH = TC_D + 4;      // floats per row of the partial result a CTA leaves in shared memory
+constexpr int TC_XO_BYTES = 2 * TC_MT * TC_XO_PITCH * 4;        // 256 rows; their (max, sum) pairs follow
+static_assert(TC_XO_BYTES + 2 * TC_MT * 8 <= (2 + 2 * TC_STAGES) * TC_TILE_BYTES, "the partial result reuses the tile buffers");
 
 // barrier slots
 enum { B_Q = 0, B_KFULL = 1, B_VFULL = 3, B_KEMPTY = 5, B_VEMPTY = 7, B_SFULL = 9, B_PFULL = 11, B_ODONE = 13 };
@@ -59,6 +62,7 @@ struct TcArgs {
   int B, N, W, Hq, Hkv, g;
   float scale_log2;
   int splits, m_blocks;
+  int cluster_merge;           // the key ranges of a (sequence, head, tile pair) form a cluster and merge in shared memory
   __nv_bfloat16 *out;
   float *part_o;
   float2 *part_ml;
@@ -196,6 +200,26 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ inline uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t *>(&v);
+}
+// ---- distributed shared memory of a thread-block cluster ----
+__device__ inline uint32_t cluster_map(uint32_t addr, uint32_t cta_rank) {     // my shared address, seen in CTA cta_rank
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta_rank));
+  return r;
+}
+__device__ inline float4 cluster_ld_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ inline float2 cluster_ld_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+// every thread of every CTA of the cluster; orders shared-memory writes before it against reads after it
+__device__ inline void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 }  // namespace
@@ -492,7 +516,30 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // in the loads, and only the stores are per lane.
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(B_ODONE + i), (nt - 1) & 1, abort_flag));
     const bool in_range = R < rows_total;
-    if (ok && __any_sync(0xFFFFFFFFu, in_range)) {
+    if (a.cluster_merge) {
+      // The key ranges of this (sequence, head, tile pair) are the CTAs of one cluster: each leaves
+      // its partial result in its own shared memory (the tile buffers are free once both query
+      // tiles' MMAs have finished, hence the barrier over the 256 softmax threads) and the merge
+      // reads them from there after the cluster barrier at the end of the kernel.
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const int rr = i * TC_MT + r_local;
+      float *xo = reinterpret_cast<float *>(gen_base) + (size_t)rr * TC_XO_PITCH;
+      float2 *xml = reinterpret_cast<float2 *>(gen_base + TC_XO_BYTES);
+      const bool dump = ok && __any_sync(0xFFFFFFFFu, in_range);     // warp-uniform; rows past the last are never read
+      if (dump) {
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < TC_D; c0 += 32) {
+          uint32_t r[32];
+          tc_ld32(t_O + c0, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            reinterpret_cast<uint4 *>(xo + c0)[c] = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+        }
+      }
+      xml[rr] = (ok && row_valid) ? make_float2(m_used, l_run) : make_float2(-CUDART_INF_F, 0.f);
+    } else if (ok && __any_sync(0xFFFFFFFFu, in_range)) {
       tc_fence_after();
       const int node = in_range ? R / a.g : 0, qh = in_range ? R - node * a.g : 0;
       if (a.splits == 1) {
@@ -547,6 +594,54 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
   tc_fence_before();
   __syncthreads();
+  if (a.cluster_merge) {
+    // ---- merge of the cluster's partial results: CTA c takes every splits-th share of the 256
+    // packed rows, one warp per row, lane l the output columns 4l..4l+3 ----
+    cluster_sync_all();
+    if (warp < 8) {
+      const int S = a.splits;
+      const int share = (2 * TC_MT + S - 1) / S;
+      const int r_lo = split * share, r_hi = min(2 * TC_MT, r_lo + share);
+      const uint32_t xo0 = smem_u32(gen_base), xml0 = smem_u32(gen_base + TC_XO_BYTES);
+      for (int rr = r_lo + warp; rr < r_hi; rr += 8) {
+        const int Rm = mpair * 2 * TC_MT + rr;
+        if (Rm >= rows_total) break;
+        const float2 ml = lane < S ? cluster_ld_f2(cluster_map(xml0 + (uint32_t)rr * 8u, (uint32_t)lane))
+                                   : make_float2(-CUDART_INF_F, 0.f);
+        float gm = ml.x;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
+        const float w = (ml.x == -CUDART_INF_F) ? 0.f : fast_exp2(ml.x - gm);    // an empty range has no row to read
+        float lsum = w * ml.y;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const uint32_t row_off = xo0 + ((uint32_t)rr * TC_XO_PITCH + (uint32_t)lane * 4u) * 4u;
+        for (int s0 = 0; s0 < S; s0 += 4) {        // the loads of four ranges go out before any is used
+          float ws[4];
+          float4 o4[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int sidx = s0 + u;
+            ws[u] = __shfl_sync(0xFFFFFFFFu, w, sidx & 31);
+            if (sidx >= S) ws[u] = 0.f;
+            o4[u] = ws[u] != 0.f ? cluster_ld_f4(cluster_map(row_off, (uint32_t)sidx)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            acc.x += ws[u] * o4[u].x; acc.y += ws[u] * o4[u].y; acc.z += ws[u] * o4[u].z; acc.w += ws[u] * o4[u].w;
+          }
+        }
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        const int node = Rm / a.g, qh = Rm - node * a.g;
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2 *>(a.out + (((int64_t)b * a.N + node) * a.Hq + kvh * a.g + qh) * TC_D + lane * 4) = packed;
+      }
+    }
+    cluster_sync_all();                    // nobody leaves while a peer may still read its shared memory
+  }
   if (warp == 9) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS) : "memory");
@@ -609,7 +704,8 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
                                  const void *kt, const void *vt, const int64_t *kv_start, const int32_t *block_table,
                                  int bt_stride, int64_t stride_t,
                                  int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
-                                 int splits, int m_blocks, cudaStream_t st) {
+                                 int splits, int m_blocks, cudaStream_t st, int *merged_in_kernel) {
+  *merged_in_kernel = 0;
   const int N = c->p.budget, Hq = c->p.n_q_heads, Hkv = c->p.n_kv_heads, g = Hq / Hkv, B = c->B;
   CUtensorMap mq, mkp, mvp, mkt, mvt;
   {
@@ -640,9 +736,45 @@ talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *
   a.out = (__nv_bfloat16 *)out; a.part_o = c->d_attn_o; a.part_ml = c->d_attn_ml; a.status = c->d_status;
   (void)max_prefix_len;
   dim3 grid((m_blocks + 1) / 2, splits, B * Hkv);
+  // Two to eight key ranges: they are launched as one thread-block cluster and merge their partial
+  // results through distributed shared memory, if the device can place such a cluster (asked once
+  // per cluster size; a cluster of full-SM CTAs needs that many SMs free in one GPC).
+  a.cluster_merge = 0;
+  // (few rows: the second kernel is cheaper than a cluster launch and two cluster barriers)
+  const long long merge_rows = (long long)B * Hkv * g * N * splits;
+  if ((c->attn_cluster == 2 || (c->attn_cluster == 1 && merge_rows >= c->attn_cluster_min_rows)) && splits >= 2 &&
+      splits <= 8) {
+    cudaLaunchConfig_t q = {};
+    q.gridDim = grid; q.blockDim = dim3(TC_THREADS); q.dynamicSmemBytes = TC_SMEM; q.stream = st;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = (unsigned)splits; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa; q.numAttrs = 1;
+    if (c->attn_cluster_ok[splits] < 0) {
+      int n = 0;
+      const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel, &q);
+      if (e != cudaSuccess) cudaGetLastError();
+      c->attn_cluster_ok[splits] = (e == cudaSuccess && n >= 1) ? 1 : 0;
+    }
+    a.cluster_merge = c->attn_cluster_ok[splits];
+  }
   {
     LaunchTimer lt(c, TALON_K_ATTENTION, st);
-    launch_kernel(c, tree_attention_tc_kernel, grid, dim3(TC_THREADS), TC_SMEM, st, mq, mkp, mvp, mkt, mvt, a);
+    if (a.cluster_merge) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = grid; cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = TC_SMEM; cfg.stream = st;
+      cudaLaunchAttribute attr[2];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)splits; attr[0].val.clusterDim.z = 1;
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = (c->pdl == 1 || (c->pdl < 0 && c->B <= PDL_AUTO_BATCH)) ? 2 : 1;
+      cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel, mq, mkp, mvp, mkt, mvt, a);
+      *merged_in_kernel = 1;
+    } else {
+      launch_kernel(c, tree_attention_tc_kernel, grid, dim3(TC_THREADS), TC_SMEM, st, mq, mkp, mvp, mkt, mvt, a);
+    }
   }
   if (cudaGetLastError() != cudaSuccess) return TALON_ERR_CUDA;
   c->launches += 1;

@@ -121,6 +121,10 @@ struct talon_ctx {
   unsigned int *d_row_count;         // [rows_cap]               chunks finished per row
   unsigned int *d_seq_count;         // [batch_max]              chunks finished per sequence (fused kernel)
   int fused_grid;                    // CTAs of the fused kernel at full width
+  int attn_cluster;                  // key ranges of the tensor-core attention merge inside a cluster (1) or in a second kernel (0)
+  long long attn_cluster_min_rows;   // automatic mode: least rows x key ranges for the merge inside the cluster
+  int attn_cluster_cap;              // more key ranges than eight are cut back to eight up to this many
+  int attn_cluster_ok[9];            // per cluster size: -1 not asked yet, 0 the device cannot place it, 1 it can
   int attn_force_splits;             // > 0: key ranges per (sequence, head, query tiles), for experiments
   int argmax_oversplit;              // target argmax: chunk rounds per CTA when the rows outnumber the grid
   int expand_max_split;              // fused kernel: chunks a row is cut into at most when the grid has room
@@ -222,7 +226,7 @@ bool attention_tc_supported(const talon_ctx *c, int64_t stride_t, int64_t stride
 talon_status launch_attention_tc(talon_ctx *c, const talon_tree *t, const void *q, const void *kp, const void *vp,
                                  const void *kt, const void *vt, const int64_t *kv_start, const int32_t *block_table,
                                  int bt_stride, int64_t stride_t, int64_t stride_h, int64_t kv_tokens, int max_prefix_len, float sm_scale, void *out,
-                                 int splits, int m_blocks, cudaStream_t st);
+                                 int splits, int m_blocks, cudaStream_t st, int *merged_in_kernel);
 talon_status launch_accept(talon_ctx *c, const talon_tree *t, const float *target_logits,
                            int64_t row_stride, int32_t *target_tok, int32_t *accept_len,
                            int32_t *accept_nodes, int32_t *bonus_tok, cudaStream_t st, bool close_tree = false);

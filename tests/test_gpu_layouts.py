@@ -119,3 +119,25 @@ def test_group_sizes_that_do_not_divide_128(hq, hkv, batch):
     assert per_step in (cfg.max_depth + 4, cfg.max_depth + 5, cfg.max_depth + 6)
     list(_check_all(cfg, t, wl, talon))
     t.close()
+
+
+@pytest.mark.parametrize("mode", ["0", "2"])
+@pytest.mark.parametrize("batch,prefix", [(1, 700), (1, 2900), (3, 1500)])
+def test_key_ranges_merged_in_a_cluster_or_by_the_second_kernel(mode, batch, prefix, monkeypatch):
+    """Few sequences: a (sequence, head) is cut into key ranges.  Their partial results are merged
+    either through the distributed shared memory of a thread-block cluster (forced here for every
+    size: 2 to 8 ranges per cluster, ragged last range, unused query tile) or by a second kernel;
+    both against the oracle, and against each other within the rounding of the final division."""
+    talon, workload = _mods()
+    monkeypatch.setenv("TALON_ATTN_CLUSTER", mode)                   # read when the context is made
+    cfg = synth.CONFIGS["tiny"].scaled(batch=batch, prefix_min=prefix, prefix_max=prefix + 130, vocab=8000)
+    t = workload.make_talon(cfg)
+    wl = workload.build_workload(cfg, t, SEED)
+    launches = t.launch_count()
+    workload.run_step(t, wl)
+    per_step = t.launch_count() - launches
+    assert t.poll_status() == talon.OK
+    list(_check_all(cfg, t, wl, talon))
+    if mode == "2":
+        assert per_step <= cfg.max_depth + 4         # reset, layers, build, attention (merged in the kernel), arg-max
+    t.close()

@@ -202,7 +202,8 @@ def test_multi_step_loop_in_one_call_matches_the_oracle_step_by_step():
                 assert torch.equal(al[s], ref_results[s][0]) and torch.equal(bo[s], ref_results[s][2])
                 assert torch.equal(an[s], ref_results[s][1])
             assert (bits(out) == bits(ref_results[-1][3])).all()
-    assert per_loop >= S * (D + 6)
+    # per step at least: reset, D layers, attention, arg-max (its last CTA walks and closes the tree), 2 for the commit
+    assert per_loop >= S * (D + 5)
     # Section 5.3's figures from the counters, against the oracle's formulas
     m = talon.loop_metrics(cnt2, 0.1)
     n_p, n_q, length = (int(x) for x in cnt2.sum(dim=0).tolist())
