@@ -3,8 +3,11 @@
 // Work split.  For sequence b and kv head h the g = Hq/Hkv query heads of all N tree nodes are
 // packed into one [g*N, 128] query matrix (row = node * g + head-in-group), so every K/V tile
 // is read once for the whole group.  A CTA owns up to two 128-row query tiles and a range of
-// 128-key tiles of the key axis (the L_b prefix keys, then the tree keys); with several
-// ranges per (b, h) a second kernel merges the partial results (split-KV).
+// 128-key tiles of the key axis (the L_b prefix keys, then the tree keys).  Several ranges per
+// (b, h) are merged either inside the kernel -- the ranges form a thread-block cluster, leave
+// their partial results in shared memory and every CTA merges a share of the rows through
+// distributed shared memory -- or, for more than eight ranges or very few rows, by a second kernel
+// from fp32 partials in global memory (split-KV).
 //
 // Roles inside a CTA (320 threads):
 //   warps 0-3, 4-7  softmax of query tile 0 / 1: thread r owns row r.  It reads its row of
